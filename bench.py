@@ -28,9 +28,18 @@ WORKLOAD = dict(name="C3", B=2, H=16, T=16384, d=128, m=128, W=64, seed=30)
 DECODE = dict(name="C5", n_seq=256, H=16, d=128, m=128, W=64, prefix=16384, steps=1024, seed=50)
 METRIC = "linsimp_fwd_bwd_tokens_per_s_T16k"
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12     # CUDA-core fp32: SMs x lanes x 2 x max clock
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch at B=2 H=16 T=4096 d=m=128 (ncu capture summarised
-# in profiles/ncu_fwd_tc_bwd_tc_small_T4096.md)
-NCU_DRAM_BYTES_T4096 = {"fwd_tc": 484.9e6, "bwd_tc": 1475.6e6}
+
+
+def ncu_dram_bytes():
+    """DRAM bytes (read + write) per launch of the tile kernels as a profiler capture of a small case counted them:
+    {"T": tokens per sequence of the captured case, "kernels": {name: bytes per launch}}, from the data file kept
+    beside the capture's summary; None when the file is missing."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_bytes_small_case.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except (OSError, ValueError):
+        return None
 
 
 def measured_peaks():
@@ -171,7 +180,7 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def bench_decode(P, synth, torch, dev, steps, warmup):
+def bench_decode(P, synth, torch, dev, steps, warmup, use_image=True, use_graph=True):
     cfg = DECODE
     n_seq, H, d, m, W = cfg["n_seq"], cfg["H"], cfg["d"], cfg["m"], cfg["W"]
     omega = synth.make_omega(d, m).to(dev)
@@ -207,14 +216,13 @@ def bench_decode(P, synth, torch, dev, steps, warmup):
                       dtype=torch.uint8, device=dev)
     # the constant feature matrix is converted once (linsimp_decode_prepare), not in every step
     wsd = P.decode_prepare(n_seq, H, d, omega, W=W)
-    use_image = os.environ.get("LS_NO_OMEGA_IMAGE") is None
     for s in range(warmup):
         q, k_, v_, r_, u_ = toks[s % pool]
         P.decode_step(q, k_, v_, r_, u_, omega, S, z, rr, ru, pos_all[s], W=W, out=out, workspace=wsd,
                       omega_image=use_image)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    graphed = os.environ.get("LS_NO_GRAPH") is None and steps % pool == 0
+    graphed = use_graph and steps % pool == 0
     if graphed:
         # `pool` consecutive steps per CUDA graph (a serving loop would do the same): the positions of the steps
         # live in one tensor that a single add advances per replay
@@ -258,6 +266,69 @@ def bench_decode(P, synth, torch, dev, steps, warmup):
                 launches_per_step=launches, finite=finite, cuda_graph=graphed, omega_image=use_image)
 
 
+def bench_secondary(P, synth, torch, dev, steps, peaks):
+    """The secondary configurations: the feature-rank sweep (C4: B=4 H=8 T=8192 d=64, m in 32..256, fwd+bwd) and the
+    layer forward (C2: B=8 H=16 T=4096 d=64 m=128).  A few timed steps each, CUDA events on the launching stream."""
+    def frac(tf):
+        return dict(frac_of_measured_bf16_burst=tf / peaks["bf16_burst"], frac_of_nominal_bf16=tf / 2250.0)
+
+    rows = []
+    for mm in (32, 64, 128, 256):
+        cfg4, t4 = synth.make_config("C4m%d" % mm)
+        g4 = {k_: v_.to(dev) for k_, v_ in t4.items()}
+        p4 = P.binding.make_params(cfg4["B"], cfg4["H"], cfg4["T"], cfg4["d"], mm, 64, P.BF16)
+        ws4 = torch.empty(max(P.workspace_bytes(p4, P.OP_BWD), P.workspace_bytes(p4, P.OP_FWD), 256),
+                          dtype=torch.uint8, device=dev)
+
+        def step4():
+            o4, L4, lse4 = P.fwd(g4["q"], g4["k"], g4["v"], g4["r"], g4["u"], g4["omega"], workspace=ws4)
+            P.bwd(g4["q"], g4["k"], g4["v"], g4["r"], g4["u"], g4["omega"], o4, L4, lse4, g4["dO"], workspace=ws4,
+                  reuse_fwd_state=True)
+
+        for _ in range(3):
+            step4()
+        torch.cuda.synchronize()
+        P.profile_enable(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step4()
+        e1.record()
+        torch.cuda.synchronize()
+        prof4 = P.profile_read()
+        P.profile_enable(False)
+        ms = e0.elapsed_time(e1) / steps
+        th4 = cfg4["B"] * cfg4["H"] * cfg4["T"]
+        fl = 3.0 * fwd_flops_per_token_head(cfg4["d"], mm, 64) * th4
+        tf = fl / (ms * 1e-3) / 1e12
+        rows.append(dict(m=mm, ms_per_step=ms, tokens_per_s=cfg4["B"] * cfg4["T"] / (ms * 1e-3), tflops_3x=tf,
+                         kernels={k_: round(v_[0] / steps, 3) for k_, v_ in prof4.items()}, **frac(tf)))
+        del g4, ws4
+    # layer forward (C2), forward only
+    cfg2, t2 = synth.make_config("C2", with_dO=False)
+    g2 = {k_: v_.to(dev) for k_, v_ in t2.items()}
+    p2 = P.binding.make_params(cfg2["B"], cfg2["H"], cfg2["T"], cfg2["d"], cfg2["m"], 64, P.BF16)
+    ws2 = torch.empty(P.workspace_bytes(p2, P.OP_FWD), dtype=torch.uint8, device=dev)
+    o2 = torch.empty_like(g2["q"])
+    for _ in range(3):
+        P.fwd(g2["q"], g2["k"], g2["v"], g2["r"], g2["u"], g2["omega"], workspace=ws2, out=o2)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        P.fwd(g2["q"], g2["k"], g2["v"], g2["r"], g2["u"], g2["omega"], workspace=ws2, out=o2)
+    e1.record()
+    torch.cuda.synchronize()
+    ms2 = e0.elapsed_time(e1) / steps
+    th2 = cfg2["B"] * cfg2["H"] * cfg2["T"]
+    tf2 = fwd_flops_per_token_head(cfg2["d"], cfg2["m"], 64) * th2 / (ms2 * 1e-3) / 1e12
+    c2 = dict(ms=ms2, tokens_per_s=cfg2["B"] * cfg2["T"] / (ms2 * 1e-3), tflops=tf2, **frac(tf2))
+    del g2, ws2, o2
+    return dict(steps=steps,
+                c4_sweep="C4: B=4 H=8 T=8192 d=64 W=64 bf16, fwd+bwd, TFLOP/s in the 3x convention", c4=rows,
+                c2_forward="C2: B=8 H=16 T=4096 d=64 m=128 bf16, fwd only", c2=c2)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -268,6 +339,9 @@ def main():
     ap.add_argument("--skip-decode", action="store_true")
     ap.add_argument("--decode-only", action="store_true", help="run only the decode benchmark (profiler captures)")
     ap.add_argument("--decode-prefix", type=int, default=DECODE["prefix"], help="prefix length used to build the decode state")
+    ap.add_argument("--no-graph", action="store_true", help="decode: launch every step instead of replaying CUDA graphs (profiler captures)")
+    ap.add_argument("--no-omega-image", action="store_true", help="decode: every step converts omega itself (profiler captures)")
+    ap.add_argument("--skip-secondary", action="store_true", help="leave out the secondary configurations (C2 forward, C4 sweep)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--small", action="store_true", help="T=4096 variant for profiler captures (not a bench value)")
@@ -331,58 +405,8 @@ def main():
                               hbm_peak_gbs=peaks["hbm_gbs"], kernels=res)))
         return
     if args.sweep:
-        rows = []
-        for mm in (32, 64, 128, 256):
-            cfg4, t4 = synth.make_config("C4m%d" % mm)
-            g4 = {k_: v_.to(dev) for k_, v_ in t4.items()}
-            p4 = P.binding.make_params(cfg4["B"], cfg4["H"], cfg4["T"], cfg4["d"], mm, 64, P.BF16)
-            ws4 = torch.empty(max(P.workspace_bytes(p4, P.OP_BWD), P.workspace_bytes(p4, P.OP_FWD), 256),
-                              dtype=torch.uint8, device=dev)
-
-            def step4():
-                o4, L4, lse4 = P.fwd(g4["q"], g4["k"], g4["v"], g4["r"], g4["u"], g4["omega"], workspace=ws4)
-                P.bwd(g4["q"], g4["k"], g4["v"], g4["r"], g4["u"], g4["omega"], o4, L4, lse4, g4["dO"], workspace=ws4,
-                      reuse_fwd_state=True)
-
-            for _ in range(3):
-                step4()
-            torch.cuda.synchronize()
-            P.profile_enable(True)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(args.steps):
-                step4()
-            e1.record()
-            torch.cuda.synchronize()
-            prof4 = P.profile_read()
-            P.profile_enable(False)
-            ms = e0.elapsed_time(e1) / args.steps
-            th4 = cfg4["B"] * cfg4["H"] * cfg4["T"]
-            fl = 3.0 * fwd_flops_per_token_head(cfg4["d"], mm, 64) * th4
-            rows.append(dict(m=mm, ms_per_step=ms, tokens_per_s=cfg4["B"] * cfg4["T"] / (ms * 1e-3),
-                             tflops_3x=fl / (ms * 1e-3) / 1e12,
-                             kernels={k_: round(v_[0] / args.steps, 3) for k_, v_ in prof4.items()}))
-            del g4, ws4
-        # layer forward (C2: B=8 H=16 T=4096 d=64 m=128), forward only
-        cfg2, t2 = synth.make_config("C2", with_dO=False)
-        g2 = {k_: v_.to(dev) for k_, v_ in t2.items()}
-        p2 = P.binding.make_params(cfg2["B"], cfg2["H"], cfg2["T"], cfg2["d"], cfg2["m"], 64, P.BF16)
-        ws2 = torch.empty(P.workspace_bytes(p2, P.OP_FWD), dtype=torch.uint8, device=dev)
-        o2 = torch.empty_like(g2["q"])
-        for _ in range(3):
-            P.fwd(g2["q"], g2["k"], g2["v"], g2["r"], g2["u"], g2["omega"], workspace=ws2, out=o2)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            P.fwd(g2["q"], g2["k"], g2["v"], g2["r"], g2["u"], g2["omega"], workspace=ws2, out=o2)
-        e1.record()
-        torch.cuda.synchronize()
-        ms2 = e0.elapsed_time(e1) / args.steps
-        th2 = cfg2["B"] * cfg2["H"] * cfg2["T"]
-        c2 = dict(ms=ms2, tokens_per_s=cfg2["B"] * cfg2["T"] / (ms2 * 1e-3),
-                  tflops=fwd_flops_per_token_head(cfg2["d"], cfg2["m"], 64) * th2 / (ms2 * 1e-3) / 1e12)
-        del g2, ws2, o2
+        sec = bench_secondary(P, synth, torch, dev, args.steps, peaks)
+        rows, c2 = sec["c4"], sec["c2"]
         # whole head on C3: normalisation with temperature -> estimator -> gated RMSNorm, and back
         cfg3, t3 = synth.make_config("C3")
         g3 = {k_: v_.to(dev) for k_, v_ in t3.items()}
@@ -418,7 +442,7 @@ def main():
                               c3_head="C3 inputs through the whole head (tau = sqrt(d), gamma = -2), fwd+bwd", c3h=c3h)))
         return
     if args.decode_only:
-        dec = bench_decode(P, synth, torch, dev, args.decode_steps, 3)
+        dec = bench_decode(P, synth, torch, dev, args.decode_steps, 3, not args.no_omega_image, not args.no_graph)
         dec["frac_hbm"] = dec["gbs"] / peaks["hbm_gbs"]
         print(json.dumps(dict(decode=dec)))
         return
@@ -556,7 +580,7 @@ def main():
 
     decode = None
     if not args.skip_decode and not args.small and rank == 0:
-        decode = bench_decode(P, synth, torch, dev, args.decode_steps, 8)
+        decode = bench_decode(P, synth, torch, dev, args.decode_steps, 8, not args.no_omega_image, not args.no_graph)
         decode["frac_hbm"] = decode["gbs"] / peaks["hbm_gbs"]
         decode["peak_gbs"] = peaks["hbm_gbs"]
         decode["peak_source"] = peaks["source"]
@@ -580,8 +604,8 @@ def main():
         "fwd_fp32": (2.0 * m * 2 * d * W * th, "alu", FP32_FMA_PEAK_TFLOPS),
         "bwd_query_fp32": (3 * 2.0 * W * m * d * th, "alu", FP32_FMA_PEAK_TFLOPS),
         "bwd_kv_fp32": (2.0 * W * m * d * th, "alu", FP32_FMA_PEAK_TFLOPS),
-        "fwd_tc": (2.0 * m * 2 * d * W * th, "tensor", peaks["bf16_sustained"]),
-        "bwd_tc": (2.0 * 2.0 * m * 2 * d * W * th, "tensor", peaks["bf16_sustained"]),
+        "fwd_tc": (2.0 * m * 2 * d * W * th, "tensor", peaks["bf16_burst"]),
+        "bwd_tc": (2.0 * 2.0 * m * 2 * d * W * th, "tensor", peaks["bf16_burst"]),
     }
     roofline = None
     if prof:
@@ -591,20 +615,29 @@ def main():
         if name in alg:
             fl, bound, peak = alg[name]
             ach = fl / (avg_ms * 1e-3) / 1e12
-            # DRAM bytes per launch from the committed ncu capture of the T=4096 case (profiles/), scaled by
-            # the number of tiles (traffic is proportional to tokens: states, images and gradients per chunk)
-            traffic = {"bwd_tc": NCU_DRAM_BYTES_T4096.get("bwd_tc"), "fwd_tc": NCU_DRAM_BYTES_T4096.get("fwd_tc")}.get(name)
-            if traffic is not None:
-                traffic = traffic * (T / 4096.0)
+            # DRAM bytes per launch: counted by a profiler capture of a smaller case of the same kernel and scaled by
+            # the tokens per sequence (the traffic - states, images and gradients per chunk - grows with the tokens)
+            cap = ncu_dram_bytes()
+            traffic = None
+            if cap and name in cap.get("kernels", {}):
+                traffic = cap["kernels"][name] * (T / float(cap["T"]))
             roofline = dict(kernel=name, bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
                             traffic=traffic, avg_ms=avg_ms, launches=cnt,
                             peak_source=("derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz" if bound == "alu"
-                                         else "of %s (sustained bf16)" % peaks["source"]))
+                                         else "of %s (burst bf16)" % peaks["source"]))
+            if bound == "tensor":
+                roofline["frac_of_sustained"] = ach / peaks["bf16_sustained"]
+                roofline["traffic_source"] = (None if traffic is None else
+                                              "profiler capture at T=%d scaled by T/%d" % (cap["T"], cap["T"]))
         else:
             roofline = dict(kernel=name, bound=None, achieved=None, peak=None, unit=None, frac=None, traffic=None,
                             avg_ms=avg_ms, launches=cnt)
     kernels = {k_: dict(ms_total=v_[0], launches=v_[1], share=v_[0] / max(1e-9, sum(x[0] for x in prof.values())))
                for k_, v_ in prof.items()}
+
+    secondary = None
+    if not args.skip_secondary and not args.small:
+        secondary = bench_secondary(P, synth, torch, dev, 5, peaks)
 
     cpu = None
     if not args.skip_cpu_baseline and world == 1:
@@ -620,7 +653,8 @@ def main():
                             parallelism="independent (batch, head) units per rank, no collective"),
                 tflops=tflops, frac_of_nominal_bf16=tflops["3x"] / (2250.0 * world),
                 frac_of_measured_bf16_sustained=tflops["3x"] / (peaks["bf16_sustained"] * world),
-                roofline=roofline, kernels=kernels, cpu_baseline=cpu, clocks=clocks,
+                frac_of_measured_bf16_burst=tflops["3x"] / (peaks["bf16_burst"] * world),
+                roofline=roofline, secondary=secondary, kernels=kernels, cpu_baseline=cpu, clocks=clocks,
                 gpu_launches=launches_per_step * args.steps, finite=finite, decode=decode,
                 attempts_ms_per_step=attempts)
     if e2e:

@@ -115,10 +115,10 @@ size_t linsimp_workspace_bytes(const linsimp_params *p, int op);
  *        rowmax_L [B,H,T] fp32   L_i of App. B.2
  *        lse      [B,H,T] fp32   L_i + log(Z'_i + eps'_i), where Z' is the shifted
  *                                normaliser without 1/m and eps' = eps*m*exp(-L_i);
- *                                i.e. log(m*(Z_i + eps)).  Both are what the
- *                                backward needs besides the inputs ("one
- *                                stabilizer scalar per query/head" plus the
- *                                log-normaliser).
+ *                                i.e. log(m*(Z_i + eps)).  rowmax_L is the per-row
+ *                                shift of App. B.2 and lse the log-normaliser; with
+ *                                the inputs they are all the backward needs
+ *                                (Sec. 4.2 "Backward").
  *        S_final [B,H,m,d], z_final [B,H,m] fp32, nullable (both or neither):
  *                                prefix state after the last token, in the
  *                                decode convention above.
@@ -348,7 +348,10 @@ int linsimp_last_launch_count(int op);
  *     LINSIMP_OP_FWD: B*H*ceil(T/32)*(m*d+m)*4 bytes) exceeds the array are refused with
  *     LINSIMP_ETOOLARGE before anything is launched.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call before starting any stream capture.
+ *     current).  With CUDA's lazy module loading that look-up is also what loads the part of
+ *     the library that holds the array, so the driver reserves the 32 MiB - and may stall for
+ *     it - inside that first call.  Make it once at start-up, outside any time-critical loop
+ *     and before starting any stream capture; later calls only read a cached address.
  *   - All calls on a device share the one array.  It keeps the previous call's contents, which
  *     is harmless: every element a call reads it has written first, so nothing needs clearing.
  *     But two calls whose kernels overlap in time on the GPU (different streams, no ordering)

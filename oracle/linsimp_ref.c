@@ -18,7 +18,7 @@
  * omega [n_omega][d][m], unit n uses bank n % n_omega; states M [m][d], a [m]
  * including the 1/sqrt(m) factor.  Rows < t0 are history: their keys/values
  * are already inside (M0,a0) and they serve only as anchors.
- * Pinned by tests against linsimp_ref.py and its pins; not "parity unpinned".
+ * Pinned by tests against linsimp_ref.py and, through it, by that file's pins.
  */
 #include <math.h>
 #include <stdlib.h>

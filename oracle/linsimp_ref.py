@@ -28,8 +28,8 @@ convergence to the exact windowed joint softmax (Eq. exact-window-app), the
 W=1/u=1 reduction to causal random-feature linear attention, the Omega=0 closed
 form, causality / convex-hull / bilinearity invariants, and for the gradients
 central finite differences, torch fp64 autograd through the brute-force form
-and the Euler identities <dv,v> = <du,u> = <dO,o>.  No function here is
-"parity unpinned".
+and the Euler identities <dv,v> = <du,u> = <dO,o>.  Every function here has
+at least one such pin.
 """
 import numpy as np
 

@@ -19,7 +19,7 @@ maps to zero.
 The gradient functions are the chain rule written out for these definitions;
 they are pinned by central finite differences of the forward functions, the
 forward functions by their defining properties (unit norm, unit mean square,
-scale invariance, hand-computed rows).  No function here is "parity unpinned".
+scale invariance, hand-computed rows).  Every function here has such a pin.
 """
 import numpy as np
 

@@ -74,7 +74,7 @@ bool params_ok(const linsimp_params *p, int op)
     if (!p) return false;
     if (p->B < 1 || p->H < 1 || p->d < 1 || p->m < 1 || p->W < 1) return false;
     if (op != LINSIMP_OP_DECODE && p->T < 1) return false;
-    if ((long long)p->B * p->H > 65535) return op == LINSIMP_OP_DECODE;   // grid.y limit of the chunked kernels
+    if (op != LINSIMP_OP_DECODE && (long long)p->B * p->H > 65535) return false;   // grid.y limit of the chunked kernels
     if (p->io_dtype != LINSIMP_F32 && p->io_dtype != LINSIMP_BF16) return false;
     if (p->algo != LINSIMP_ALGO_DEFAULT && p->algo != LINSIMP_ALGO_FP32) return false;
     if (!(p->eps >= 0.f)) return false;
@@ -126,9 +126,13 @@ int norm_workspace_check(const linsimp_params *p, const void *workspace, size_t 
 
 int decode_banks(const linsimp_params *p) { return p->omega_per_head ? p->H : 1; }
 
+// A shape is served either by the CUDA-core kernels (any io_dtype and algo) or, for feature ranks above 128, by the
+// tensor-core feature blocks, which exist for bf16 I/O with the default algo only.
 bool shape_supported(const linsimp_params *p)
 {
-    return p->W <= 64 && (simt_supported(p->d, p->m) || tc_blocks_supported(p->d, p->m));
+    if (p->W > 64) return false;
+    if (simt_supported(p->d, p->m)) return true;
+    return p->io_dtype == LINSIMP_BF16 && p->algo == LINSIMP_ALGO_DEFAULT && tc_blocks_supported(p->d, p->m);
 }
 
 // feature ranks above 128 (bf16 I/O, default algo): several 128-feature column blocks on the tensor-core kernels
@@ -283,7 +287,7 @@ int run_tc(const linsimp_params *p, const void *q, const void *k, const void *v,
         const TcLayout LB = tc_layout(p, LINSIMP_OP_BWD);
         if (workspace_bytes >= LB.total) a.chi32 = (float *)(ws + LB.chi32);
     }
-    cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream);
+    if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
     const int op = state_only ? LINSIMP_OP_STATE : LINSIMP_OP_FWD;
     return finish(op, tc_fwd_run(a, (cudaStream_t)stream));
 }
@@ -321,7 +325,7 @@ int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void
     a.dchi_intra = (float *)(tws + TL.dchi_intra);
     a.dr_acc = (float *)(tws + TL.dr_acc);
     a.du_acc = (float *)(tws + TL.du_acc);
-    cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream);
+    if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
     return finish(LINSIMP_OP_BWD, tc_bwd_run(a, (cudaStream_t)stream));
 }
 
@@ -365,7 +369,7 @@ int run_tc_blocks(int op, const linsimp_params *p, const void *q, const void *k,
         a.dr_acc = (float *)(ws + L.dr_acc);
         a.du_acc = (float *)(ws + L.du_acc);
     }
-    cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream);
+    if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
     TcBlockWs bw;
     tc_blocks_carve(ws + base, p->B, p->H, p->T, p->d, p->m, op, &bw);
     const float lem = log_eps_m(p);

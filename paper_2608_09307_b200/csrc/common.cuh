@@ -39,4 +39,13 @@ struct Shape {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Streaming multiprocessors of the current device (launch heuristics size their grids by it); 148 if the query fails.
+inline int sm_count()
+{
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 148;
+    return n;
+}
+
 }  // namespace linsimp

@@ -501,10 +501,10 @@ k_decode_mma(const bf16 *__restrict__ q, const bf16 *__restrict__ k, const bf16 
     }
 }
 
-// banks: 1 (one Omega for all heads) or H (one per head; every CTA then serves one head, which needs H <= 148)
+// banks: 1 (one Omega for all heads) or H (one per head; every CTA then serves one head, which needs H <= the SM count)
 int decode_mma_supported(int d, int m, int W, int banks)
 {
-    return (d == 64 || d == 128) && (m == 64 || m == 128) && W <= DW && W >= 1 && banks <= 148;
+    return (d == 64 || d == 128) && (m == 64 || m == 128) && W <= DW && W >= 1 && banks <= sm_count();
 }
 
 size_t decode_mma_image_bytes(int d, int m, int banks) { return 2 * (size_t)m * (d + 8) * 2 * banks; }
@@ -534,8 +534,9 @@ static int decode_run_t(const SimtArgs &a, const void *omega_image, cudaStream_t
     LaunchScope sc = {st, 0};
     sc.check(cudaFuncSetAttribute(k_decode_mma<DD, DM>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::TOTAL));
     const int per_head = a.omega_stride != 0 && a.H > 1;
-    int grid = n_units < 148 ? n_units : 148;
-    if (per_head) grid = (grid / a.H) * a.H;               // a multiple of H (n_units is one, and H <= 148)
+    const int sms = sm_count();
+    int grid = n_units < sms ? n_units : sms;
+    if (per_head) grid = (grid / a.H) * a.H;               // a multiple of H (n_units is one, and H <= the SM count)
     const float log2_eps_m = a.log_eps_m * 1.4426950408889634f;
     LS_LAUNCH(sc, "decode_mma", k_decode_mma<DD, DM><<<grid, 512, SM::TOTAL, st>>>(
         (const bf16 *)a.q, (const bf16 *)a.k, (const bf16 *)a.v, (const bf16 *)a.r, (const bf16 *)a.u, a.omega, a.H, a.W,

@@ -1574,8 +1574,8 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
     LS_LAUNCH(sc, "omega_image_tc", k_omega_image_pad_tc<D, MF><<<n_om, 256, 0, st>>>(a.omega, a.m_real, a.omega_ld,
                                                                                      a.omega_stride, a.om_img));
     if (!a.keep_acc) {
-        cudaMemsetAsync(a.dr_acc, 0, sizeof(float) * ntok, st);
-        cudaMemsetAsync(a.du_acc, 0, sizeof(float) * ntok, st);
+        sc.check(cudaMemsetAsync(a.dr_acc, 0, sizeof(float) * ntok, st));
+        sc.check(cudaMemsetAsync(a.du_acc, 0, sizeof(float) * ntok, st));
     }
     const int smem = S::TOTAL + 1024;
     const int cpc = a.chunks_per_cta;
@@ -1594,7 +1594,8 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
     else launch(k_bwd_tc<D, MF, 0>);
     // Segments of the key/value sweep: one wave of CTAs (two per SM) where the sequence is long enough, never shorter
     // than KV_SEG chunks (the workspace holds one partial sum per KV_SEG chunks).
-    const int want = (2 * 148) / BH > 0 ? (2 * 148) / BH : 1;
+    const int slots = 2 * sm_count();
+    const int want = slots / BH > 0 ? slots / BH : 1;
     int seg_len = (NC + want - 1) / want;
     if (seg_len < KV_SEG) seg_len = KV_SEG;
     const int NSEG = (NC + seg_len - 1) / seg_len;

@@ -87,12 +87,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // Bounded wait: every wait in this library gives up after kWaitLimit polls, records the
 // failure in *status (device memory, may be null) and lets the kernel run to its end.
 static constexpr uint32_t kWaitLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int code)
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, int *status, int code, uint32_t limit)
 {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     if (status) atomicExch(status, code);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int *status, int code)
+{
+    return mbar_wait_limit(bar, parity, status, code, kWaitLimit);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -1,22 +1,16 @@
 // Bring-up probe for the tcgen05 path: runs one accumulation chain of UMMA instructions on
 // operand images and descriptors supplied by the caller and returns the fp32 accumulator.
 // Used by the GPU tests to pin the descriptor encodings and the swizzled operand layouts
-// the production kernels rely on.  Not part of the public header.
+// the production kernels rely on.  Only the encodings those kernels build are accepted: anything
+// else is refused on the host, so that no unchecked descriptor ever reaches the tensor cores.
+// A second probe exercises the give-up path of the bounded waits.  Declared in linsimp_debug.h.
+#include "../../include/linsimp_debug.h"
 #include "common.cuh"
 #include "tc_common.cuh"
 
 namespace linsimp {
 
-struct UmmaProbe {
-    uint32_t idesc;
-    uint32_t a_lbo, a_sbo, a_layout;
-    uint32_t b_lbo, b_sbo, b_layout;
-    int nk;
-    int a_koff[16], b_koff[16];   // byte offsets added to the operand start address per K step
-    int a_bytes, b_bytes;         // image sizes (multiples of 16)
-    int n_out;                    // accumulator columns to read back (multiple of 16, <= 256)
-    int a_from_tmem;              // A image is [128][a_bytes/512] 32-bit words per row, stored to TMEM
-};
+typedef linsimp_umma_probe UmmaProbe;
 
 __global__ void __launch_bounds__(128) k_umma_probe(const uint4 *__restrict__ a_img, const uint4 *__restrict__ b_img,
                                                     UmmaProbe pr, float *__restrict__ out, int *status)
@@ -88,12 +82,80 @@ __global__ void __launch_bounds__(128) k_umma_probe(const uint4 *__restrict__ a_
 
 }  // namespace linsimp
 
-extern "C" int linsimp_debug_umma(const void *a_img, const void *b_img, const linsimp::UmmaProbe *probe, float *out,
+namespace linsimp {
+
+// A test-only kernel whose single wait can never succeed: the barrier expects one arrival and nothing arrives.  After
+// `limit` polls the wait gives up, records `code` in *status and the kernel returns without touching the barrier,
+// tensor memory or any copy engine again - the path every production kernel takes when one of its waits runs out.
+__global__ void k_wait_expiry(int *status, int code, uint32_t limit, int *polled)
+{
+    using namespace tc;
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const bool ok = mbar_wait_limit(&bar, 0, status, code, limit);
+        if (polled) *polled = ok ? 0 : 1;
+    }
+}
+
+namespace {
+// the instruction descriptors the production kernels build: kind::f16 with an fp32 accumulator, both operands of the
+// same 16-bit format, M = 128, N a multiple of 16 up to 256, either operand K-major or MN-major
+bool idesc_known(uint32_t d)
+{
+    const uint32_t fa = (d >> 7) & 7u, fb = (d >> 10) & 7u, n8 = (d >> 17) & 0x3Fu, m16 = (d >> 24) & 0x1Fu;
+    const uint32_t known = (1u << 4) | (7u << 7) | (7u << 10) | (1u << 15) | (1u << 16) | (0x3Fu << 17) | (0x1Fu << 24);
+    if (d & ~known) return false;
+    if (!(d & (1u << 4))) return false;
+    if (fa != fb || fa > 1u) return false;
+    if (m16 != 8u) return false;
+    return n8 >= 2u && n8 <= 32u && (n8 & 1u) == 0u;
+}
+// shared-memory operands: a swizzled layout the kernels use, strides in whole 16-byte units, every K step inside the image
+bool operand_known(uint32_t lbo, uint32_t sbo, uint32_t layout, const int *koff, int nk, int bytes)
+{
+    if (!(layout == tc::kSw128 || layout == tc::kSw64 || layout == tc::kSw32)) return false;
+    if ((lbo & 15u) || (sbo & 15u) || lbo > (1u << 18) || sbo > (1u << 18) || sbo == 0) return false;
+    if (bytes < 512 || (bytes & 15)) return false;
+    for (int k = 0; k < nk; ++k)
+        if (koff[k] < 0 || (koff[k] & 15) || koff[k] >= bytes) return false;
+    return true;
+}
+}  // namespace
+}  // namespace linsimp
+
+extern "C" int linsimp_debug_wait_expiry(int *status, int code, unsigned limit, int *gave_up, void *stream)
+{
+    using namespace linsimp;
+    if (!status || code <= 0 || limit < 1 || limit > (1u << 16)) return -1;
+    k_wait_expiry<<<1, 32, 0, (cudaStream_t)stream>>>(status, code, limit, gave_up);
+    return cudaPeekAtLastError() == cudaSuccess ? 0 : -5;
+}
+
+extern "C" int linsimp_debug_umma(const void *a_img, const void *b_img, const linsimp_umma_probe *probe, float *out,
                                   int *status, void *stream)
 {
     using namespace linsimp;
     if (!a_img || !b_img || !probe || !out) return -1;
     if (probe->nk < 1 || probe->nk > 16 || probe->n_out < 16 || probe->n_out > 256 || probe->n_out % 16) return -1;
+    if (probe->a_bytes < 512 || probe->b_bytes < 512 || (probe->a_bytes & 15) || (probe->b_bytes & 15)) return -1;
+    if (!idesc_known(probe->idesc)) return -2;
+    if ((int)(((probe->idesc >> 17) & 0x3Fu) << 3) < probe->n_out) return -2;     // reads only columns the product wrote
+    if (!operand_known(probe->b_lbo, probe->b_sbo, probe->b_layout, probe->b_koff, probe->nk, probe->b_bytes)) return -2;
+    if (probe->a_from_tmem) {
+        // A is [128][words] 32-bit words stored to tensor memory behind the accumulator: K-major only, steps inside it
+        const int words = probe->a_bytes / 512;
+        if ((probe->idesc >> 15) & 1u) return -2;
+        if (words < 8 || words > 256 || (words & 31)) return -2;
+        for (int k = 0; k < probe->nk; ++k)
+            if (probe->a_koff[k] < 0 || probe->a_koff[k] + 8 > words) return -2;
+    } else if (!operand_known(probe->a_lbo, probe->a_sbo, probe->a_layout, probe->a_koff, probe->nk, probe->a_bytes)) {
+        return -2;
+    }
     const size_t smem = 1024 + ((probe->a_bytes + 1023) & ~1023) + ((probe->b_bytes + 1023) & ~1023);
     if (smem > 200 * 1024) return -1;
     if (cudaFuncSetAttribute(k_umma_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return -5;

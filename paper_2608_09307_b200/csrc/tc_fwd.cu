@@ -872,7 +872,7 @@ static int fwd_tc_impl(const TcArgs &a, cudaStream_t st)
     using SS = StateSmem<D, MF>;
     // segments of the state walk: as many as fill the two CTA slots of every SM, at most kStateSegMax, none for short
     // sequences
-    int n_seg = (2 * 148) / (BH * (MF / 64));
+    int n_seg = (2 * sm_count()) / (BH * (MF / 64));
     if (n_seg > kStateSegMax) n_seg = kStateSegMax;
     if (n_seg > NC / 32) n_seg = NC / 32;
     if (n_seg < 1) n_seg = 1;

@@ -1,18 +1,10 @@
 """Multi-GPU host logic: the path shards over independent (batch, head) units with no data-path
-collective; the only communication is the host-side agreement on timing (max over ranks).
+collective - every rank runs its own batch of the same shape (weak scaling) - and the only
+communication is the host-side agreement on timing (max over ranks) and the total of the units.
 
 One process per GPU (torch.distributed; NCCL on GPUs, gloo in the CPU tests)."""
 import torch
 import torch.distributed as dist
-
-
-def shard_units(n_units, world_size, rank):
-    """Contiguous, balanced split of `n_units` independent (batch, head) units: returns (begin, end)."""
-    if world_size < 1 or not (0 <= rank < world_size):
-        raise ValueError("bad world_size/rank")
-    base, rem = divmod(n_units, world_size)
-    begin = rank * base + min(rank, rem)
-    return begin, begin + base + (1 if rank < rem else 0)
 
 
 def max_over_ranks(value, device="cpu"):

@@ -1,5 +1,6 @@
-"""Host-side multi-process logic on CPU (gloo, world_size 2): unit sharding is a partition and the
-timing agreement is the max over ranks.  No GPU and no data-path collective is involved."""
+"""Host-side multi-process logic on CPU (gloo, world_size 2): every rank runs its own units, the step time
+is the max over ranks and the job's throughput the units of all ranks over that time.  No GPU and no
+data-path collective is involved."""
 import os
 import socket
 
@@ -7,18 +8,7 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2608_09307_b200.dist import aggregate_throughput, max_over_ranks, shard_units
-
-
-def test_shard_units_is_a_partition():
-    for n in (1, 7, 32, 33, 4096):
-        for w in (1, 2, 3, 8):
-            cuts = [shard_units(n, w, r) for r in range(w)]
-            assert cuts[0][0] == 0 and cuts[-1][1] == n
-            for a, b in zip(cuts, cuts[1:]):
-                assert a[1] == b[0]
-            sizes = [e - b for b, e in cuts]
-            assert max(sizes) - min(sizes) <= 1
+from paper_2608_09307_b200.dist import aggregate_throughput, max_over_ranks
 
 
 def _free_port():
@@ -34,11 +24,11 @@ def _worker(rank, world, port, out):
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     try:
-        b, e = shard_units(33, world, rank)
+        units = 16 + rank                                 # the ranks' own batches
         step_ms = 10.0 + 5.0 * rank                       # rank 1 is the slow one
         tmax = max_over_ranks(step_ms)
-        thr = aggregate_throughput(e - b, tmax * 1e-3)
-        out.put((rank, b, e, tmax, thr))
+        thr = aggregate_throughput(units, tmax * 1e-3)
+        out.put((rank, units, tmax, thr))
     finally:
         dist.destroy_process_group()
 
@@ -55,6 +45,6 @@ def test_two_ranks_agree_on_max_time_and_total_throughput():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    assert [r[1:3] for r in res] == [(0, 17), (17, 33)]
-    assert all(abs(r[3] - 15.0) < 1e-9 for r in res)       # max over ranks
-    assert all(abs(r[4] - 33 / 15e-3) < 1e-6 for r in res) # all units / slowest time
+    assert [r[1] for r in res] == [16, 17]
+    assert all(abs(r[2] - 15.0) < 1e-9 for r in res)       # max over ranks
+    assert all(abs(r[3] - 33 / 15e-3) < 1e-6 for r in res) # all units / slowest time

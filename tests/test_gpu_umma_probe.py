@@ -149,3 +149,55 @@ def test_a_from_tmem():
         pr.b_koff[k] = (k // 4) * N * 128 + (k % 4) * 32
     out = run(i16(A).reshape(-1), kmajor_image(i16(B), 128), pr, N)
     assert np.abs(out - ref).max() < 2e-2 * np.abs(ref).max()
+
+
+def test_unknown_descriptors_are_refused_before_launch():
+    """The probe accepts only the encodings the production kernels build."""
+    lib = P.load_library()
+    A, B, _ = mats(128, 128, 128, torch.bfloat16, 6)
+    a = torch.from_numpy(kmajor_image(i16(A), 128).copy()).cuda()
+    b = torch.from_numpy(kmajor_image(i16(B), 128).copy()).cuda()
+    out = torch.zeros(128, 128, device="cuda")
+
+    def call(mutate):
+        pr = Probe()
+        pr.idesc = idesc(128, 128, 1, 0, 0)
+        pr.a_lbo, pr.a_sbo, pr.a_layout = 0, 1024, SW[128]
+        pr.b_lbo, pr.b_sbo, pr.b_layout = 0, 1024, SW[128]
+        pr.nk = 8
+        for k in range(8):
+            pr.a_koff[k] = pr.b_koff[k] = (k // 4) * 128 * 128 + (k % 4) * 32
+        pr.a_bytes, pr.b_bytes, pr.n_out = a.numel() * 2, b.numel() * 2, 128
+        mutate(pr)
+        return lib.linsimp_debug_umma(ctypes.c_void_p(a.data_ptr()), ctypes.c_void_p(b.data_ptr()), ctypes.byref(pr),
+                                      ctypes.c_void_p(out.data_ptr()), None, None)
+
+    assert call(lambda pr: None) == 0
+    torch.cuda.synchronize()
+    mixed = (1 << 4) | (0 << 7) | (1 << 10) | (16 << 17) | (8 << 24)          # fp16 A with bf16 B: no such product
+    for bad in (lambda pr: setattr(pr, "idesc", mixed),
+                lambda pr: setattr(pr, "idesc", idesc(64, 128, 1, 0, 0)),       # M = 64
+                lambda pr: setattr(pr, "idesc", idesc(128, 128, 1, 0, 0) | (1 << 2)),   # a reserved bit
+                lambda pr: setattr(pr, "idesc", idesc(128, 24, 1, 0, 0)),       # N not a multiple of 16
+                lambda pr: setattr(pr, "a_layout", 1),
+                lambda pr: setattr(pr, "b_sbo", 1000),
+                lambda pr: pr.b_koff.__setitem__(7, pr.b_bytes)):               # a K step beyond the image
+        assert call(bad) == -2
+    torch.cuda.synchronize()
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait nothing ever satisfies runs out after its poll limit: the kernel returns, the status word holds the
+    wait's code, and the context keeps working (a product afterwards is correct)."""
+    lib = P.load_library()
+    status = torch.zeros(64, dtype=torch.int32, device="cuda")     # laid out like the head of a workspace
+    gave_up = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert lib.linsimp_read_status(ctypes.c_void_p(status.data_ptr()), None) == 0
+    rc = lib.linsimp_debug_wait_expiry(ctypes.c_void_p(status.data_ptr()), 77, 4096, ctypes.c_void_p(gave_up.data_ptr()), None)
+    assert rc == 0
+    assert lib.linsimp_read_status(ctypes.c_void_p(status.data_ptr()), None) == 77      # synchronises the stream
+    assert int(gave_up.item()) == 1
+    assert lib.linsimp_debug_wait_expiry(ctypes.c_void_p(status.data_ptr()), 0, 4096, None, None) == -1
+    assert lib.linsimp_debug_wait_expiry(ctypes.c_void_p(status.data_ptr()), 5, 1 << 20, None, None) == -1
+    # the device is healthy afterwards
+    test_kmajor_sw128(torch.bfloat16, 1, 128, 128)

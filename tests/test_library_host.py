@@ -86,6 +86,58 @@ def test_workspace_and_argument_checks_on_host():
     assert lib.linsimp_ring_fill_padded(ctypes.byref(p), al, al, n, al, al, n) == -1
 
 
+def test_large_decode_batches_still_get_every_check():
+    """More than 65535 (sequence, head) units are fine for the decode step (its grid does not depend on them), and
+    the remaining parameter checks apply to such a batch like to any other."""
+    lib = P.load_library()
+    n = ctypes.c_void_p(None)
+    big = binding.make_params(8192, 16, 0, 128, 128, 64, P.BF16)
+    assert lib.linsimp_decode_step(ctypes.byref(big), *([n] * 13), 0, n) == -1        # null pointers, not the size
+    assert P.workspace_bytes(big, P.OP_DECODE) > 0
+    assert P.workspace_bytes(big, P.OP_FWD) == 0                                       # the chunked kernels' grid limit
+    for field, value in (("io_dtype", 7), ("eps", float("nan")), ("eps", -1.0), ("flags", 64), ("algo", 9)):
+        bad = binding.make_params(8192, 16, 0, 128, 128, 64, P.BF16)
+        setattr(bad, field, value)
+        assert P.workspace_bytes(bad, P.OP_DECODE) == 0, field
+        buf = ctypes.create_string_buffer(4096)
+        al = ctypes.c_void_p((ctypes.addressof(buf) + 255) // 256 * 256)
+        assert lib.linsimp_decode_step(ctypes.byref(bad), *([al] * 13), 1 << 20, n) == -1, field
+
+
+def test_workspace_is_zero_where_no_kernel_serves_the_combination():
+    # feature ranks above 128 exist as tensor-core feature blocks for bf16 I/O with the default algo only
+    ok = binding.make_params(1, 2, 100, 128, 256, 64, P.BF16)
+    assert P.workspace_bytes(ok, P.OP_FWD) > 0
+    for io, algo in ((P.F32, P.ALGO_DEFAULT), (P.BF16, P.ALGO_FP32), (P.F32, P.ALGO_FP32)):
+        none = binding.make_params(1, 2, 100, 128, 256, 64, io, False, algo)
+        assert P.workspace_bytes(none, P.OP_FWD) == 0
+        assert P.workspace_bytes(none, P.OP_BWD) == 0
+    # d = 64 has a CUDA-core instance at m = 256
+    assert P.workspace_bytes(binding.make_params(1, 2, 100, 64, 256, 64, P.F32), P.OP_FWD) > 0
+
+
+def test_descriptor_probe_refuses_unknown_encodings_on_the_host():
+    lib = P.load_library()
+
+    class Probe(ctypes.Structure):
+        _fields_ = [("idesc", ctypes.c_uint32),
+                    ("a_lbo", ctypes.c_uint32), ("a_sbo", ctypes.c_uint32), ("a_layout", ctypes.c_uint32),
+                    ("b_lbo", ctypes.c_uint32), ("b_sbo", ctypes.c_uint32), ("b_layout", ctypes.c_uint32),
+                    ("nk", ctypes.c_int), ("a_koff", ctypes.c_int * 16), ("b_koff", ctypes.c_int * 16),
+                    ("a_bytes", ctypes.c_int), ("b_bytes", ctypes.c_int), ("n_out", ctypes.c_int),
+                    ("a_from_tmem", ctypes.c_int)]
+
+    pr = Probe()
+    pr.idesc = (1 << 4) | (0 << 7) | (1 << 10) | (16 << 17) | (8 << 24)                 # fp16 A with bf16 B
+    pr.a_lbo, pr.a_sbo, pr.a_layout = 0, 1024, 2
+    pr.b_lbo, pr.b_sbo, pr.b_layout = 0, 1024, 2
+    pr.nk, pr.a_bytes, pr.b_bytes, pr.n_out = 1, 32768, 32768, 128
+    buf = ctypes.create_string_buffer(64)
+    al = ctypes.c_void_p(ctypes.addressof(buf))
+    assert lib.linsimp_debug_umma(al, al, ctypes.byref(pr), al, None, None) == -2         # refused before any launch
+    assert lib.linsimp_debug_wait_expiry(None, 1, 100, None, None) == -1
+
+
 def test_ops_refuse_cpu_tensors():
     import pytest
     import torch
