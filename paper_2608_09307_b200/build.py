@@ -30,6 +30,7 @@ def build_library(force=False, verbose=False):
     nvcc = os.environ.get("NVCC", "nvcc")
     os.makedirs(OBJ, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
+    extra += os.environ.get("LINSIMP_NVCC_EXTRA", "").split()        # e.g. -DLS_FWD_TRACE for a tuning build
 
     def compile_one(src):
         obj = os.path.join(OBJ, src[:-3] + ".o")

@@ -14,8 +14,9 @@
 // with psi' = exp(l - L_i) written to shared memory as bf16 between GEMM-1 and GEMM-2.
 // GEMM-2 is computed transposed so that a thread owns one output channel e and sums the
 // anchors with plain FMAs against u_c[e]; only the scalar normaliser needs a warp-shuffle
-// reduction.  Each of the two warpgroups owns a private TMEM region and runs its tiles
-// start to finish; the two overlap each other's tensor and SFU phases.
+// reduction.  The kernel is warp-specialised: row warps (composite queries, exponentials, masks), a product warp
+// that issues every tensor-core instruction, channel warps (anchor sums, output) and a load warp hand tiles to one
+// another through mbarriers, two tiles in flight on two sets of tensor-memory and shared-memory buffers.
 #include "common.cuh"
 #include "launch.cuh"
 #include "tc_common.cuh"
@@ -27,8 +28,6 @@ namespace linsimp {
 using namespace tc;
 
 static constexpr int TC_C = kTcChunk;       // tokens per chunk
-static constexpr int TC_SLOTS = 2;          // tiles in flight per CTA
-static constexpr int TC_NT = TC_SLOTS * 256;
 
 // ------------------------------------------------------------------ image geometry
 // all byte sizes; MF in {64,128}, D in {64,128}
@@ -480,37 +479,80 @@ __device__ __forceinline__ float2 unpack_bf16(uint32_t w)
     return __bfloat1622float2(v);
 }
 
+// ---- shared-memory map of the main kernel
 template <int D, int MF>
-struct FwdTcSmem {
+struct FwdWsSmem {
     using G = TcGeom<D, MF>;
-    static constexpr int WROWS = 5 * TC_C;                        // anchor window: ring of 5 groups of 16 tokens
+    static constexpr int RING = 6 * TC_C;                         // anchor rows r: ring of 6 groups of 16 tokens
     static constexpr int ROWB = D * 2;                            // bytes per token row
-    static constexpr int PITCH = ROWB + 16;                       // window row pitch (conflict-free 16-byte row reads)
     static constexpr int OFF_OM = 0;
-    static constexpr int OFF_CHUNK0 = OFF_OM + G::IMG_OM;
-    static constexpr int OFF_CHUNK1 = OFF_CHUNK0 + G::IMG_CHUNK;
-    static constexpr int OFF_PSI = OFF_CHUNK1 + G::IMG_CHUNK;     // per tile slot: [128][MF] bf16
+    static constexpr int OFF_IMG = OFF_OM + G::IMG_OM;            // two chunk images
+    static constexpr int OFF_PSI = OFF_IMG + 2 * G::IMG_CHUNK;    // per tile buffer: [128][MF] bf16
     static constexpr int PSI_BYTES = 128 * MF * 2;
-    static constexpr int OFF_PM = OFF_PSI + TC_SLOTS * PSI_BYTES; // per tile slot: [128][16] bf16 (32-byte rows)
+    static constexpr int OFF_PM = OFF_PSI + 2 * PSI_BYTES;        // per tile buffer: [128][16] bf16 (32-byte rows)
     static constexpr int PM_BYTES = 128 * 32;
-    static constexpr int OFF_RWIN = OFF_PM + TC_SLOTS * PM_BYTES; // [WROWS][D] fp16, padded rows
-    static constexpr int OFF_Q = OFF_RWIN + ((WROWS * PITCH + 1023) / 1024) * 1024;
-    static constexpr int OFF_AB = OFF_Q + TC_C * ROWB;            // [MF] fp32
-    static constexpr int OFF_HN = OFF_AB + MF * 4;                // per slot: [2 halves][128] fp32 partial |x|^2/2
-    static constexpr int OFF_ACC = OFF_HN + TC_SLOTS * 2 * 128 * 4;   // per slot: [2 halves][2 queries][128] fp32 partial N
-    static constexpr int OFF_MISC = OFF_ACC + TC_SLOTS * 4 * 128 * 4; // per slot: 8 warp maxima, 8 warp sums, 2 L, 2 den
-    static constexpr int TOTAL = OFF_MISC + TC_SLOTS * 128;
+    static constexpr int OFF_RWIN = OFF_PM + 2 * PM_BYTES;        // [RING][D] fp16, 16-byte pieces swizzled by row
+    static constexpr int OFF_Q = OFF_RWIN + RING * ROWB;          // two chunks of [16][D] fp16
+    static constexpr int OFF_AB = OFF_Q + 2 * TC_C * ROWB;        // two chunks of [MF] fp32
+    static constexpr int OFF_HN = OFF_AB + 2 * MF * 4;            // per tile buffer: [2 tiles][2 halves][128] fp32 partial |x|^2/2
+    static constexpr int OFF_MISC = OFF_HN + 2 * 2 * 2 * 128 * 4; // per tile buffer 32 floats, see below
+    static constexpr int TOTAL = OFF_MISC + 2 * 32 * 4;
 };
 
-// grid (ceil(NC / chunks_per_cta), B*H), 512 threads = 2 tile slots x 2 column halves x 128 rows.
-// A tile is 128 composite rows = 2 queries x 64 steps back; each slot works through every second tile of the
-// chunk, so that the products of one slot run under the CUDA-core phases of the other.  The two threads of a
-// row own half of the feature columns each (rows side) and half of the steps back each (channel side).
-// MODE 1 (HIST): the segment continues a sequence (anchors of the n_hist tokens before it come from hist_r, hist_u);
-// the plain instance carries no trace of it.  MODE 2 (O32): `o` points to an fp32 buffer (the output of one feature
-// block, to be combined with the other blocks' in full precision).
+// TMEM column map of the main kernel (512 allocated): per tile buffer the composite queries X (fp16 pairs, the A operand
+// of the first product), the 128-column accumulator that holds l and then Dt, the intra-chunk pair weights P; and the
+// channel warps' private window of u (bf16 pairs, written twice 40 columns apart so that any 33 consecutive pairs are
+// contiguous).
+static constexpr uint32_t WS_X = 0, WS_L = 128, WS_P = 384, WS_U = 416;
+#ifndef LS_FWD_RS
+#define LS_FWD_RS 2
+#endif
+#ifndef LS_FWD_XE
+#define LS_FWD_XE 0
+#endif
+#ifndef LS_FWD_P1
+#define LS_FWD_P1 16       // columns requested per wait in the maximum pass
+#endif
+#ifndef LS_FWD_P2
+#define LS_FWD_P2 0        // 1: the exponential pass requests the next piece before working on the current one
+#endif
+static constexpr int WS_RS = LS_FWD_RS;        // threads per tile row in the row warps (1 or 2)
+static constexpr int WS_GW = 4 * WS_RS;        // warps of one row group
+static constexpr int WS_CW0 = 2 * WS_GW;       // first channel warp; then the product warp and the load warp
+static constexpr int WS_NT = (WS_CW0 + 8) * 32;   // (the last warpgroup: product warp, load warp, two idle warps)
+
+// Bounded wait that also ends when another role of the CTA has already given up (`*abort` set): after one wait of the
+// pipeline has run out, every other wait returns at once and the kernel runs to its end with undefined results.
+__device__ __forceinline__ void ws_wait(uint64_t *bar, uint32_t parity, int *status, int code, volatile int *abort)
+{
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((i & 255u) == 255u && *abort) return;
+    }
+    *abort = 1;
+    if (status) atomicExch(status, code);
+}
+__device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t &r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+}
+
+// grid (ceil(NC / chunks_per_cta), B*H), WS_NT threads in five roles that hand tiles to one another through mbarriers.
+// A tile is 128 composite rows = 2 queries x 64 steps back; tiles alternate between two sets of buffers, so that the
+// products of one tile run under the CUDA-core stages of its neighbours:
+//   row warps (two groups of eight, one group per buffer; two threads per tile row, half of the columns each):
+//       X = q_i * r_c (fp16) into tensor memory, row maximum L_i, psi' = exp(l - L_i) as a bf16 operand tile with the
+//       row's part of the normaliser, causal mask of the intra-chunk pair weights; the next tile's X is formed while
+//       the pair weights of the current one are being computed;
+//   product warp (one thread): l = X . OmegaT;  P = psi' . chi'^T;  Dt = MbT . psi'^T + Vt . Pm^T  (transposed, so that a
+//       channel owns a tensor-memory lane);
+//   channel warps (thread = output channel e): N_i[e] = sum_c Dt[e,(i,c)] u_c[e] with u from a private window in
+//       tensor memory, normaliser and guard, output;
+//   load warp: chunk operand images by bulk copy, the chunk's r and q rows (converted to fp16) and boundary normaliser.
+// MODE 1 (HIST): the segment continues a sequence (anchors of the n_hist tokens before it come from hist_r, hist_u).
+// MODE 2 (O32): `o` points to an fp32 buffer (the output of one feature block, to be combined with the other blocks').
 template <int D, int MF, int MODE>
-__global__ void __launch_bounds__(TC_NT, 1)
+__global__ void __launch_bounds__(WS_NT, 1)
 k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__restrict__ u,
          const uint8_t *__restrict__ om_img, int om_per_head, int H, int T, int W, int NC, int chunks_per_cta,
          float log2_eps_m, const uint8_t *__restrict__ images, const float *__restrict__ ab_g, bf16 *__restrict__ o,
@@ -520,334 +562,508 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
     constexpr bool HIST = MODE == 1, O32 = MODE == 2;
     const int n_hist = HIST ? n_hist_arg : 0;
     using G = TcGeom<D, MF>;
-    using S = FwdTcSmem<D, MF>;
+    using S = FwdWsSmem<D, MF>;
     constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
-    constexpr int CH = D / 8;                     // 16-byte chunks per token row
-    constexpr int XW = D / 4;                     // packed fp16 words of X per thread (half a row)
-    constexpr int FH = MF / 2;                    // feature columns per thread
+    constexpr int CH = D / 8;                     // 16-byte pieces per token row
+    constexpr int XW = D / 2;                     // packed fp16 words of X per row
+    constexpr int NT = TC_C / 2;                  // tiles per chunk
     extern __shared__ __align__(1024) uint8_t smem_dyn[];
     // 1024-byte alignment by an offset into the array (not by pointer casts), so that accesses stay shared-space loads/stores
     uint8_t *smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-    __shared__ uint64_t bar_full[2], bar_om, bar_mma[TC_SLOTS][3];
+    // per tile buffer: X written, l ready, psi' written, P ready, Pm written, Dt ready, accumulator read by the channels
+    __shared__ uint64_t bar_x[2], bar_l[2], bar_psi[2], bar_p[2], bar_pm[2], bar_dt[2], bar_free[2];
+    // per chunk parity: image arrived, image no longer read, rows (r, q, a_b) written, rows no longer read
+    __shared__ uint64_t bar_img[2], bar_imgfree[2], bar_rows[2], bar_rowsfree[2], bar_om;
     __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int slot = tid >> 8, hf = (tid >> 7) & 1, t = tid & 127;   // t = tile row (rows side) / channel (epilogue)
-    const int wis = (warp & 3) + 4 * hf;                             // warp index inside the slot
     const int bh = blockIdx.y;
     const int n_begin = blockIdx.x * chunks_per_cta;
     const int n_end = min(NC, n_begin + chunks_per_cta);
     const long seq_off = (long)bh * T * D;
 
-    if (warp == 0) {
+    if (warp == WS_CW0 + 4) {
         tmem_alloc(&tmem_base_s, 512);
         tmem_relinquish();
     }
     if (tid == 0) {
-        mbar_init(&bar_full[0], 1);
-        mbar_init(&bar_full[1], 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bar_x[b], WS_GW);
+            mbar_init(&bar_l[b], 1);
+            mbar_init(&bar_psi[b], WS_GW);
+            mbar_init(&bar_p[b], 1);
+            mbar_init(&bar_pm[b], WS_GW);
+            mbar_init(&bar_dt[b], 1);
+            mbar_init(&bar_free[b], 4);
+            mbar_init(&bar_img[b], 1);
+            mbar_init(&bar_imgfree[b], 1);
+            mbar_init(&bar_rows[b], 1);
+            mbar_init(&bar_rowsfree[b], 2 * WS_GW);
+        }
         mbar_init(&bar_om, 1);
-        for (int g = 0; g < TC_SLOTS; ++g)
-            for (int x = 0; x < 3; ++x) mbar_init(&bar_mma[g][x], 1);
+        abort_s = 0;
         fence_barrier_init();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_sl = tmem_base_s + slot * 256;
+    const uint32_t tm = tmem_base_s;
     const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-    constexpr uint32_t TM_X = 0, TM_L = 64, TM_P = 192;     // column offsets inside the slot's region
+    volatile int *abort = &abort_s;
 
-    const uint8_t *img_bh = images + (long)bh * NC * G::IMG_CHUNK;
-    if (tid == 0) {
-        mbar_arrive_expect_tx(&bar_om, G::IMG_OM);
-        bulk_g2s(smem + S::OFF_OM, om_img + (long)(om_per_head ? bh % H : 0) * G::IMG_OM, G::IMG_OM, &bar_om);
-        mbar_arrive_expect_tx(&bar_full[0], G::IMG_CHUNK);
-        bulk_g2s(smem + S::OFF_CHUNK0, img_bh + (long)n_begin * G::IMG_CHUNK, G::IMG_CHUNK, &bar_full[0]);
-    }
-    mbar_wait(&bar_om, 0, status, 10);
-
-    uint8_t *psi_s = smem + S::OFF_PSI + slot * S::PSI_BYTES;
-    uint8_t *pm_s = smem + S::OFF_PM + slot * S::PM_BYTES;
     uint8_t *rwin = smem + S::OFF_RWIN;
-    uint8_t *qs = smem + S::OFF_Q;
-    float *abs_ = (float *)(smem + S::OFF_AB);
-    float *hnp = (float *)(smem + S::OFF_HN) + slot * 256;           // [2][128]
-    float *accp = (float *)(smem + S::OFF_ACC) + slot * 512;         // [2 halves][2 queries][128]
-    float *misc = (float *)(smem + S::OFF_MISC) + slot * 32;         // [0..7] warp max, [8..15] warp sums, [16..17] L, [18..19] den
+    float *misc_all = (float *)(smem + S::OFF_MISC);       // per buffer: [0..15] warp maxima (two sets), [16..23] warp sums, [24..25] L_i
+    const uint8_t *img_bh = images + (long)bh * NC * G::IMG_CHUNK;
+    // ring row of token `tok` (tok >= -96): the window of a chunk spans five groups, the sixth takes the next chunk's rows
+    auto ring_row = [](int tok) { return (tok + S::RING) % S::RING; };
 
-    const uint32_t idesc_1 = make_idesc_f16(128, MF, 0, 0, 0);        // fp16: X . OmegaT
-    const uint32_t idesc_p = make_idesc_f16(128, TC_C, 1, 0, 0);      // bf16: psi . chi'
-    const uint32_t idesc_2 = make_idesc_f16(128, 128, 1, 0, 0);       // bf16: MbT . psi, Vt . Pm
-    uint32_t mma_phase = 0;                                           // flips once per tile (each barrier used once per tile)
-    const bool issuer = (hf == 0) && (t == 0);                        // the slot's product-issuing thread
-
-    for (int n = n_begin; n < n_end; ++n) {
-        const int it = n - n_begin, buf = it & 1;
-        uint8_t *chunk_s = smem + (buf ? S::OFF_CHUNK1 : S::OFF_CHUNK0);
-        if (tid == 0 && n + 1 < n_end) {
-            mbar_arrive_expect_tx(&bar_full[buf ^ 1], G::IMG_CHUNK);
-            bulk_g2s(smem + (buf ? S::OFF_CHUNK0 : S::OFF_CHUNK1), img_bh + (long)(n + 1) * G::IMG_CHUNK, G::IMG_CHUNK,
-                     &bar_full[buf ^ 1]);
-            // the next chunk's token rows are read with plain loads at its start: have them in L2 by then
-            const int rows = min(TC_C, T - (n + 1) * TC_C);
-            bulk_prefetch_l2(r + seq_off + (long)(n + 1) * TC_C * D, rows * D * 2);
-            bulk_prefetch_l2(q + seq_off + (long)(n + 1) * TC_C * D, rows * D * 2);
-            bulk_prefetch_l2(u + seq_off + (long)(n + 1) * TC_C * D, rows * D * 2);      // (the epilogues read u from global memory)
-        }
-        // anchor window (a ring of five 16-token groups: group g of the sequence sits in ring slot g mod 5; the
-        // chunk needs groups n-4 .. n, of which all but group n are still there), query rows, boundary normaliser
-        const int b5 = (n + 1) % 5;                          // ring slot of group n - 4
-        auto ring_row = [&](int c) {                         // ring row of token c, c in groups n-4 .. n
-            int sl = (c >> 4) - (n - 4) + b5;
-            sl -= (sl >= 5) ? 5 : 0;
-            return sl * TC_C + (c & 15);
-        };
-        {
-            const int g_lo = (it == 0) ? n - 4 : n;
-            const int nitem = (n - g_lo + 1) * TC_C * CH;
-            for (int idx = tid; idx < nitem; idx += TC_NT) {
-                const int row = idx / CH, ch = idx - row * CH;
-                const int tok = g_lo * TC_C + row;
-                uint4 val = make_uint4(0, 0, 0, 0);
-                if (tok >= 0 && tok < T) val = *(const uint4 *)(r + seq_off + (long)tok * D + ch * 8);
-                else if (HIST && tok < 0 && tok >= -n_hist)      // anchors from before the segment
-                    val = *(const uint4 *)(hist_r + ((long)bh * n_hist + n_hist + tok) * D + ch * 8);
-                // fp16 copies (exact for bf16 values in the fp16 range): X = q * r is then one packed multiply
-                *(uint4 *)(rwin + ring_row(tok) * S::PITCH + (ch << 4)) = make_uint4(bf2h_(val.x), bf2h_(val.y), bf2h_(val.z), bf2h_(val.w));
-            }
-        }
-        {
-            const int j = (tid + TC_NT / 2) & (TC_NT - 1);   // the other half of the CTA
-            if (j < TC_C * CH) {
-                const int row = j / CH, ch = j - row * CH;
-                const int tok = n * TC_C + row;
-                uint4 val = make_uint4(0, 0, 0, 0);
-                if (tok < T) val = *(const uint4 *)(q + seq_off + (long)tok * D + ch * 8);
-                *(uint4 *)(qs + row * S::ROWB + (ch << 4)) = make_uint4(bf2h_(val.x), bf2h_(val.y), bf2h_(val.z), bf2h_(val.w));
-            }
-        }
-        for (int p = tid; p < MF; p += TC_NT) abs_[p] = ab_g[((long)bh * NC + n) * MF + p];
-        mbar_wait(&bar_full[buf], (it >> 1) & 1, status, 11);
-        __syncthreads();
-
-        const uint32_t mbt_addr = smem_u32(chunk_s);
-        const uint32_t chi_addr = mbt_addr + G::IMG_M;
-        const uint32_t vt_addr = chi_addr + G::IMG_CHI;
-
-        for (int tile = slot; tile < TC_C / 2; tile += TC_SLOTS) {
-            const int il = tile * 2 + (t >> 6);           // query index inside the chunk
-            const int i = n * TC_C + il;                  // query token
-            const int s = t & 63;                         // steps back
-            const bool valid = (s < W) && (i - s >= -n_hist) && (i < T);
-            // ---- X = q_i * r_c (fp16) into TMEM (this thread's half of the row), |x|^2/2 in fp32
-            {
-                float2 hn2 = make_float2(0.f, 0.f);
-                const int wrow = ring_row(i - s);                        // always inside the window
-                const uint8_t *rrow = rwin + wrow * S::PITCH;
-                const uint8_t *qrow = qs + il * S::ROWB;
-                uint32_t xr[XW];
+    if (warp < WS_CW0) {
+        // ================================================================== row warps
+        const int b = warp / WS_GW;                        // tile buffer of this group
+        const int w8 = warp % WS_GW;                       // warp inside the group
+        const int row = (w8 & 3) * 32 + lane;              // tile row = TMEM lane
+        const int hf = w8 >> 2;                            // which half of the row's columns
+        const int qi = row >> 6, s = row & 63;             // query of the tile, steps back
+        constexpr int FH = MF / WS_RS;                     // feature columns per thread
+        constexpr int XH = XW / WS_RS;                     // packed words of X per thread
+        float *misc = misc_all + b * 32;
+        float *hnp = (float *)(smem + S::OFF_HN) + b * 512;             // [2 tiles][2 halves][128]
+        uint8_t *psi_s = smem + S::OFF_PSI + b * S::PSI_BYTES;
+        uint8_t *pm_s = smem + S::OFF_PM + b * S::PM_BYTES;
+        // X = q_i * r_c (fp16) of tile `tile` of chunk n into tensor memory (this thread's half of the row), its part of
+        // |x|^2/2 into shared memory
+        auto make_x = [&](int n, int tile, uint32_t kk) {
+            const int c = n - n_begin;
+            const uint8_t *qs = smem + S::OFF_Q + (c & 1) * (TC_C * S::ROWB);
+            const int il = tile * 2 + qi;
+            const int rr = ring_row(n * TC_C + il - s);
+            const uint8_t *rrow = rwin + rr * S::ROWB;
+            const uint8_t *qrow = qs + il * S::ROWB;
+            float2 hn2 = make_float2(0.f, 0.f), hn3 = make_float2(0.f, 0.f);
 #pragma unroll
-                for (int c8 = 0; c8 < CH / 2; ++c8) {
-                    const int ch = hf * (CH / 2) + c8;
-                    const uint4 rv = *(const uint4 *)(rrow + (ch << 4));
+            for (int x16 = 0; x16 < XH / 16; ++x16) {
+                uint32_t xr[16];
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    const int ch = hf * (XH / 4) + x16 * 4 + c8;
+                    const uint4 rv = *(const uint4 *)(rrow + ((ch ^ (rr & 7)) << 4));
                     const uint4 qv = *(const uint4 *)(qrow + (ch << 4));
                     const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w}, qw[4] = {qv.x, qv.y, qv.z, qv.w};
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
                         const __half2 xv = __hmul2(*(const __half2 *)&rw[x], *(const __half2 *)&qw[x]);
                         const float2 xf = __half22float2(xv);
-                        hn2 = ffma2(xf, xf, hn2);
+                        if (x & 1) hn3 = ffma2(xf, xf, hn3);
+                        else hn2 = ffma2(xf, xf, hn2);
                         xr[c8 * 4 + x] = *(const uint32_t *)&xv;
                     }
                 }
-                if (XW == 32) tmem_st32(tmem_sl + lane_off + TM_X + hf * XW, (const uint32_t(&)[32])xr);
-                else tmem_st16(tmem_sl + lane_off + TM_X + hf * XW, (const uint32_t(&)[16])xr);
-                hnp[hf * 128 + t] = 0.5f * (hn2.x + hn2.y);
+                tmem_st16(tm + lane_off + WS_X + b * 64 + hf * XH + x16 * 16, xr);
             }
+            hn2 = fadd2(hn2, hn3);
+            hnp[((kk & 1) * 2 + hf) * 128 + row] = 0.5f * (hn2.x + hn2.y);
             tmem_st_wait();
             tc_fence_before();
-            bar_sync(1 + slot, 256);
-            if (issuer) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_x[b]);
+        };
+        uint32_t k = 0;                                    // tiles this group has worked on
+        ws_wait(&bar_rows[0], 0, status, 10, abort);
+        if (n_begin < n_end) make_x(n_begin, b, 0);
+        for (int n = n_begin; n < n_end; ++n) {
+            const int c = n - n_begin;
+            const float *abs_ = (const float *)(smem + S::OFF_AB) + (c & 1) * MF;
+            for (int tile = b; tile < NT; tile += 2, ++k) {
+                const int il = tile * 2 + qi;              // query index inside the chunk
+                const int i = n * TC_C + il;               // query token
+                const bool valid = (s < W) && (i - s >= -n_hist) && (i < T);
+                ws_wait(&bar_l[b], k & 1, status, 12, abort);
                 tc_fence_after();
-                const uint64_t dom = make_smem_desc(smem_u32(smem + S::OFF_OM), 0, 1024, kSw128);
+                const float hn = hnp[((k & 1) * 2) * 128 + row] + (WS_RS == 2 ? hnp[((k & 1) * 2 + 1) * 128 + row] : 0.f);
+                // ---- maximum of l = l_raw - |x|^2/2 over this thread's columns, then the query's over its 64 rows (four warps)
+                float mx = -INFINITY;
+                {
+                    // (all of this thread's columns are requested before the one wait: a tensor-memory round trip per
+                    // piece would dominate the pass)
+                    constexpr int PW = FH > LS_FWD_P1 ? LS_FWD_P1 : FH;  // columns per batch of loads
+                    float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_f16_ts(tmem_sl + TM_L, tmem_sl + TM_X + ks * 8, desc_adv(dom, (ks >> 2) * (MF * 128) + (ks & 3) * 32), idesc_1,
-                               ks > 0);
-                tc_commit(&bar_mma[slot][0]);
-            }
-            const float hn = hnp[t] + hnp[128 + t];
-            mbar_wait(&bar_mma[slot][0], mma_phase, status, 12);
-            tc_fence_after();
-            // ---- max of l = l_raw - |x|^2/2 over this thread's columns, then the query's max over its 64 rows
-            // (this thread's FH columns are read once and kept in registers for the exponentials below)
-            float mx = -INFINITY;
-            uint32_t lv[FH];
+                    for (int c0 = 0; c0 < FH; c0 += PW) {
+                        uint32_t lv[PW];
 #pragma unroll
-            for (int c0 = 0; c0 < FH; c0 += 32) tmem_ld32(tmem_sl + lane_off + TM_L + hf * FH + c0, (uint32_t(&)[32])lv[c0]);
-            tmem_ld_wait();
-            if (m_real == MF) {
+                        for (int c1 = 0; c1 < PW; c1 += 16)
+                            tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0 + c1, (uint32_t(&)[16])lv[c1]);
+                        tmem_ld_wait();
 #pragma unroll
-                for (int x = 0; x < FH; ++x) mx = fmaxf(mx, __uint_as_float(lv[x]));
-            } else {                                              // zero-padded features take no part in L_i
-#pragma unroll
-                for (int x = 0; x < FH; ++x)
-                    if (hf * FH + x < m_real) mx = fmaxf(mx, __uint_as_float(lv[x]));
-            }
-            mx = valid ? mx - hn : -INFINITY;
-            mx = warp_max(mx);
-            if (lane == 0) misc[wis] = mx;
-            bar_sync(1 + slot, 256);
-            const int qi = t >> 6;
-            float L = fmaxf(fmaxf(misc[2 * qi], misc[2 * qi + 1]), fmaxf(misc[4 + 2 * qi], misc[5 + 2 * qi]));
-            if (!(L > -INFINITY)) L = 0.f;                        // query beyond T: nothing valid
-            // ---- psi' = exp(l - L) -> bf16 tile in shared memory; zeta = psi' . a_b
-            const float shift = valid ? (hn + L) * LOG2E : INFINITY;   // invalid rows: exp2(-inf) = 0
-            float2 zeta2 = make_float2(0.f, 0.f);
-            const float2 l2e = make_float2(LOG2E, LOG2E), nshift = make_float2(-shift, -shift);
-#pragma unroll
-            for (int c0 = 0; c0 < FH; c0 += 32) {
-                const uint32_t *v = lv + c0;
-#pragma unroll
-                for (int c8 = 0; c8 < 4; ++c8) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const int col = hf * FH + c0 + c8 * 8 + x * 2;
-                        const float2 arg = ffma2(make_float2(__uint_as_float(v[c8 * 8 + x * 2]), __uint_as_float(v[c8 * 8 + x * 2 + 1])), l2e, nshift);
-                        // every fourth pair on the FMA pipes instead of the special-function unit (measured: none 4.93 ms, an eighth 4.89 ms, a quarter
-                        // 4.87 ms, half 4.97 ms on the benchmark step)
-                        const float2 pp = (x == 3) ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
-                        zeta2 = ffma2(pp, *(const float2 *)(abs_ + col), zeta2);
-                        pk[x] = pack_bf16(pp.x, pp.y);
+                        for (int x = 0; x < PW; ++x)
+                            if (m_real == MF || hf * FH + c0 + x < m_real)       // zero-padded features take no part in L_i
+                                m4[x & 3] = fmaxf(m4[x & 3], __uint_as_float(lv[x]));
                     }
-                    const int c8g = ((hf * FH + c0) >> 3) + c8;   // 8-feature chunk index over all MF
-                    *(uint4 *)(psi_s + (c8g >> 3) * (128 * 128) + sw_off<128>(t, c8g & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 }
-            }
-            float zeta = zeta2.x + zeta2.y;
-            fence_proxy_async_smem();
-            tc_fence_before();
-            bar_sync(1 + slot, 256);
-            if (issuer) {
+                mx = valid ? mx - hn : -INFINITY;
+                mx = warp_max(mx);
+                if (lane == 0) misc[(k & 1) * 8 + w8] = mx;
+                bar_sync(1 + b * 2 + qi, 64 * WS_RS);
+                const float *mq = misc + (k & 1) * 8 + 2 * qi;
+                float L = fmaxf(mq[0], mq[1]);
+                if (WS_RS == 2) L = fmaxf(L, fmaxf(mq[4], mq[5]));
+                if (!(L > -INFINITY)) L = 0.f;             // nothing valid (query beyond T)
+                // the psi' and Pm tiles of this buffer were last read by the products of the tile two before
+                if (k > 0) ws_wait(&bar_dt[b], (k - 1) & 1, status, 13, abort);
+                // ---- psi' = exp(l - L) -> bf16 operand tile; zeta = psi' . a_b
+                const float shift = valid ? (hn + L) * LOG2E : INFINITY;   // invalid rows: exp2(-inf) = 0
+                const float2 l2e = make_float2(LOG2E, LOG2E), nshift = make_float2(-shift, -shift);
+                float2 zeta2 = make_float2(0.f, 0.f), zeta3 = make_float2(0.f, 0.f);
+                {
+                    // pieces of 16 columns; the next piece is requested before the current one is worked on
+                    uint32_t lv[2][16];
+                    if (LS_FWD_P2) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH, lv[0]);
+#pragma unroll
+                    for (int pc = 0; pc < FH / 16; ++pc) {
+                        const int c0 = pc * 16;
+                        if (!LS_FWD_P2) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0, lv[0]);
+                        tmem_ld_wait();
+                        if (LS_FWD_P2 && pc + 1 < FH / 16) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0 + 16, lv[(pc + 1) & 1]);
+                        const uint32_t *lc = lv[LS_FWD_P2 ? (pc & 1) : 0];
+#pragma unroll
+                        for (int c8 = 0; c8 < 2; ++c8) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                const int col = hf * FH + c0 + c8 * 8 + x * 2;
+                                const float2 arg = ffma2(make_float2(__uint_as_float(lc[c8 * 8 + x * 2]), __uint_as_float(lc[c8 * 8 + x * 2 + 1])), l2e, nshift);
+                                // every fourth pair as a polynomial on the FMA pipes, the rest on the special-function unit
+                                const float2 pp = (x == 3) ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+                                if (x & 1) zeta3 = ffma2(pp, *(const float2 *)(abs_ + col), zeta3);
+                                else zeta2 = ffma2(pp, *(const float2 *)(abs_ + col), zeta2);
+                                pk[x] = pack_bf16(pp.x, pp.y);
+                            }
+                            const int c8g = ((hf * FH + c0) >> 3) + c8;    // 8-feature piece over all MF
+                            *(uint4 *)(psi_s + (c8g >> 3) * (128 * 128) + sw_off<128>(row, c8g & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                }
+                zeta2 = fadd2(zeta2, zeta3);
+                float zeta = zeta2.x + zeta2.y;
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&bar_psi[b]);
+                    // the last tile of the chunk for this group: its r, q rows and a_b are not read again
+                    if (tile + 2 >= NT) mbar_arrive(&bar_rowsfree[c & 1]);
+                }
+                // ---- the next tile's X (either here, while the pair weights of this one are being computed, or after the mask)
+                if (LS_FWD_XE) {
+                    if (tile + 2 < NT) {
+                        make_x(n, tile + 2, k + 1);
+                    } else if (n + 1 < n_end) {
+                        ws_wait(&bar_rows[(c + 1) & 1], ((c + 1) >> 1) & 1, status, 10, abort);
+                        make_x(n + 1, b, k + 1);
+                    }
+                }
+                // ---- intra-chunk pair weights (this thread's 8 tokens): mask j <= i, add to the normaliser, hand back as bf16
+                ws_wait(&bar_p[b], k & 1, status, 14, abort);
                 tc_fence_after();
-                const uint64_t dpsi = make_smem_desc(smem_u32(psi_s), 0, 1024, kSw128);
-                const uint64_t dchi = make_smem_desc(chi_addr, 0, 1024, kSw128), dmb = make_smem_desc(mbt_addr, 0, 1024, kSw128);
+                {
+                    constexpr int PC = TC_C / WS_RS;       // pair-weight columns per thread
+                    uint32_t v[PC];
+                    if (PC == 16) tmem_ld16(tm + lane_off + WS_P + b * 16, (uint32_t(&)[16])v);
+                    else tmem_ld8(tm + lane_off + WS_P + b * 16 + hf * 8, (uint32_t(&)[8])v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int ks = 0; ks < MF / 16; ++ks)
-                    mma_f16_ss(tmem_sl + TM_P, desc_adv(dpsi, (ks >> 2) * (128 * 128) + (ks & 3) * 32),
-                               desc_adv(dchi, (ks >> 2) * (TC_C * 128) + (ks & 3) * 32), idesc_p, ks > 0);
-                tc_commit(&bar_mma[slot][1]);
+                    for (int pc = 0; pc < PC / 8; ++pc) {
+                        uint32_t pk[4];
 #pragma unroll
-                for (int ks = 0; ks < MF / 16; ++ks) {
-                    const uint32_t koff = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
-                    mma_f16_ss(tmem_sl + TM_L, desc_adv(dmb, koff), desc_adv(dpsi, koff), idesc_2, ks > 0);
-                }
-            }
-            // ---- intra-chunk pair weights (this thread's 8 tokens): mask j <= i, add to the normaliser, hand back as bf16
-            mbar_wait(&bar_mma[slot][1], mma_phase, status, 13);
-            tc_fence_after();
-            {
-                uint32_t v[8];
-                tmem_ld8(tmem_sl + lane_off + TM_P + hf * 8, v);
-                tmem_ld_wait();
-                uint32_t pk[4];
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    const int j0 = hf * 8 + 2 * x;
-                    const float p0 = (j0 <= il) ? __uint_as_float(v[2 * x]) : 0.f;
-                    const float p1 = (j0 + 1 <= il) ? __uint_as_float(v[2 * x + 1]) : 0.f;
-                    zeta += p0 + p1;
-                    pk[x] = pack_bf16(p0, p1);
-                }
-                *(uint4 *)(pm_s + sw_off<32>(t, hf)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-            zeta = warp_sum(zeta);
-            if (lane == 0) misc[8 + wis] = zeta;
-            fence_proxy_async_smem();
-            tc_fence_before();
-            bar_sync(1 + slot, 256);
-            if (issuer) {
-                tc_fence_after();
-                const uint64_t ad = make_smem_desc(vt_addr, 0, 256, kSw32);
-                const uint64_t bd = make_smem_desc(smem_u32(pm_s), 0, 256, kSw32);
-                mma_f16_ss(tmem_sl + TM_L, ad, bd, idesc_2, 1);
-                tc_commit(&bar_mma[slot][2]);
-            }
-            if (hf == 1 && t < 2) {
-                // the query's stabiliser, normaliser and guard: den = Z' + eps*m*exp(-L)
-                const float Lq = fmaxf(fmaxf(misc[2 * t], misc[2 * t + 1]), fmaxf(misc[4 + 2 * t], misc[5 + 2 * t]));
-                const float Lf = (Lq > -INFINITY) ? Lq : 0.f;
-                const float Z = (misc[8 + 2 * t] + misc[9 + 2 * t]) + (misc[12 + 2 * t] + misc[13 + 2 * t]);
-                const float den = fmaxf(Z + ex2_approx(log2_eps_m - Lf * LOG2E), 1e-37f);
-                misc[16 + t] = Lf;
-                misc[18 + t] = den;
-            }
-            mbar_wait(&bar_mma[slot][2], mma_phase, status, 14);
-            tc_fence_after();
-            // ---- epilogue: thread = output channel e = t, steps back [32 hf, 32 hf + 32) of both queries
-            const int i0 = n * TC_C + tile * 2;
-            if (t < D) {
-                // The two queries of the tile share their anchors: anchor i0 - s is column s of query 0 and column
-                // s + 1 of query 1, so every u_c[e] is loaded once for both.
-                const int s0 = 32 * hf;
-                const bool interior = (i0 - 63 >= 0) && (i0 + 1 < T);   // every anchor row exists: no clamping
-                const bf16 *ubase = u + seq_off + (long)(i0 + 1 - s0) * D + t;
-                float acc0 = 0.f, acc1 = 0.f;
-                // (rows outside the sequence and its history have psi' = 0: any finite u will do there)
-                auto u_at = [&](int tok) {
-                    if (HIST && tok < 0 && tok >= -n_hist) return hist_u[((long)bh * n_hist + n_hist + tok) * D + t];
-                    return u[seq_off + (long)min(max(tok, 0), T - 1) * D + t];
-                };
-                uint32_t v0[32], v1[32];
-                tmem_ld32(tmem_sl + lane_off + TM_L + s0, v0);
-                tmem_ld32(tmem_sl + lane_off + TM_L + 64 + s0, v1);
-                tmem_ld_wait();
-                if (interior) {
-                    float un = __bfloat162float(ubase[0]);
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const float uj = __bfloat162float(ubase[-(x + 1) * D]);
-                        acc1 = fmaf(__uint_as_float(v1[x]), un, acc1);
-                        acc0 = fmaf(__uint_as_float(v0[x]), uj, acc0);
-                        un = uj;
-                    }
-                } else {
-                    float un = __bfloat162float(u_at(i0 + 1 - s0));
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const float uj = __bfloat162float(u_at(i0 - (s0 + x)));
-                        acc1 = fmaf(__uint_as_float(v1[x]), un, acc1);
-                        acc0 = fmaf(__uint_as_float(v0[x]), uj, acc0);
-                        un = uj;
+                        for (int x = 0; x < 4; ++x) {
+                            const int j0 = hf * PC + pc * 8 + 2 * x;
+                            const float p0 = (j0 <= il) ? __uint_as_float(v[pc * 8 + 2 * x]) : 0.f;
+                            const float p1 = (j0 + 1 <= il) ? __uint_as_float(v[pc * 8 + 2 * x + 1]) : 0.f;
+                            zeta += p0 + p1;
+                            pk[x] = pack_bf16(p0, p1);
+                        }
+                        *(uint4 *)(pm_s + sw_off<32>(row, hf * (PC / 8) + pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
-                accp[(hf * 2 + 0) * 128 + t] = acc0;
-                accp[(hf * 2 + 1) * 128 + t] = acc1;
-            }
-            tc_fence_before();
-            bar_sync(1 + slot, 256);                              // partial sums and misc[16..19] visible; L region read
-            if (t < D) {
-                const int iq = i0 + hf;                           // half hf finishes query hf
-                if (iq < T) {
-                    const float den = misc[18 + hf];
-                    const float oval = (accp[hf * 128 + t] + accp[(2 + hf) * 128 + t]) / den;
-                    if (O32) ((float *)o)[seq_off + (long)iq * D + t] = oval;
-                    else o[seq_off + (long)iq * D + t] = __float2bfloat16_rn(oval);
-                    if (t == 0) {
-                        Lout[(long)bh * T + iq] = misc[16 + hf];
-                        lse[(long)bh * T + iq] = misc[16 + hf] + LN2 * log2f(den);
+                zeta = warp_sum(zeta);
+                if (lane == 0) {
+                    misc[16 + w8] = zeta;
+                    if ((w8 & 5) == 0) misc[24 + qi] = L;    // warps 0 and 2 of the group: queries 0 and 1
+                }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_pm[b]);
+                if (!LS_FWD_XE) {
+                    if (tile + 2 < NT) {
+                        make_x(n, tile + 2, k + 1);
+                    } else if (n + 1 < n_end) {
+                        ws_wait(&bar_rows[(c + 1) & 1], ((c + 1) >> 1) & 1, status, 10, abort);
+                        make_x(n + 1, b, k + 1);
                     }
                 }
             }
-            mma_phase ^= 1;
         }
-        __syncthreads();
+    } else if (warp < WS_CW0 + 4) {
+        // ================================================================== channel warps
+        const int e = (warp & 3) * 32 + lane;              // output channel = TMEM lane
+        const bool live = e < D;
+        auto u_at = [&](int tok) -> uint32_t {             // bf16 bits of u[tok][e]; rows outside the sequence: zero
+            if (!live) return 0u;
+            if (tok >= 0 && tok < T) return (uint32_t)__bfloat16_as_ushort(u[seq_off + (long)tok * D + e]);
+            if (HIST && tok < 0 && tok >= -n_hist) return (uint32_t)__bfloat16_as_ushort(hist_u[((long)bh * n_hist + n_hist + tok) * D + e]);
+            return 0u;
+        };
+        uint32_t upf[8];                                   // the next group's 16 values, packed in token pairs
+        auto fetch_group = [&](int grp) {
+#pragma unroll
+            for (int x = 0; x < 8; ++x) upf[x] = u_at(grp * TC_C + 2 * x) | (u_at(grp * TC_C + 2 * x + 1) << 16);
+        };
+        auto store_group = [&](int grp) {                  // ring position of group grp: 8 columns, mirrored 40 further
+            const uint32_t col = 8u * (uint32_t)((grp + 10) % 5);
+            tmem_st8(tm + lane_off + WS_U + col, upf);
+            tmem_st8(tm + lane_off + WS_U + 40 + col, upf);
+        };
+        for (int grp = n_begin - 4; grp < n_begin; ++grp) {
+            fetch_group(grp);
+            store_group(grp);
+        }
+        fetch_group(n_begin);
+        for (int n = n_begin; n < n_end; ++n) {
+            const int c = n - n_begin;
+            store_group(n);
+            tmem_st_wait();
+            if (n + 1 < n_end) fetch_group(n + 1);
+            for (int tile = 0; tile < NT; ++tile) {
+                const int g = c * NT + tile, b = g & 1;
+                const uint32_t k = (uint32_t)g >> 1;
+                const int i0 = n * TC_C + tile * 2;
+                ws_wait(&bar_dt[b], k & 1, status, 15, abort);
+                tc_fence_after();
+                const float *misc = misc_all + b * 32;
+                const float L0 = misc[24], L1 = misc[25];
+                // (warps 0, 1, 4, 5 of the row group hold query 0, warps 2, 3, 6, 7 query 1)
+                float Z0 = misc[16] + misc[17], Z1 = misc[18] + misc[19];
+                if (WS_RS == 2) {
+                    Z0 += misc[20] + misc[21];
+                    Z1 += misc[22] + misc[23];
+                }
+                // the guard of the normaliser: den = Z' + eps*m*exp(-L)
+                const float den0 = fmaxf(Z0 + ex2_approx(log2_eps_m - L0 * LOG2E), 1e-37f);
+                const float den1 = fmaxf(Z1 + ex2_approx(log2_eps_m - L1 * LOG2E), 1e-37f);
+                // Pair j (j = 0..32) of the window holds the anchors (i0 - 2j, i0 - 2j + 1) =: (lo, hi).  Query i0 meets lo at
+                // step 2j and hi at step 2j - 1, query i0 + 1 meets lo at step 2j + 1 and hi at step 2j.  Column x of
+                // `w0` below is step x - 1 of query i0 (loaded one column early so that (hi, lo) pairs line up).
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                const uint32_t ucol = tm + lane_off + WS_U + 8u * (uint32_t)((n - 4 + 10) % 5) + tile;   // pair i0/2 - 32
+                const uint32_t dcol = tm + lane_off + WS_L + b * 128;
+#pragma unroll
+                for (int hq = 0; hq < 4; ++hq) {
+                    // steps 16 hq .. 16 hq + 15 of both queries: pairs j = 8 hq .. 8 hq + 7 = window columns 32 - j
+                    uint32_t w0[16], w1[16], uu[8];
+                    tmem_ld16(dcol + 16 * hq - 1, w0);
+                    tmem_ld16(dcol + 64 + 16 * hq, w1);
+                    tmem_ld8(ucol + 32 - 8 * hq - 7, uu);             // columns 32 - (8 hq + 7) .. 32 - 8 hq
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const uint32_t wd = uu[7 - jj];               // pair j = 8 hq + jj
+                        const float2 hl = make_float2(__uint_as_float(wd & 0xffff0000u), __uint_as_float(wd << 16));   // (hi, lo)
+                        acc1 = ffma2(make_float2(__uint_as_float(w1[2 * jj]), __uint_as_float(w1[2 * jj + 1])), hl, acc1);
+                        if (hq == 0 && jj == 0) acc0.y = fmaf(__uint_as_float(w0[1]), hl.y, acc0.y);   // step -1 does not exist
+                        else acc0 = ffma2(make_float2(__uint_as_float(w0[2 * jj]), __uint_as_float(w0[2 * jj + 1])), hl, acc0);
+                    }
+                }
+                {
+                    // pair j = 32: its hi anchor is step 63 of query i0
+                    uint32_t last, ulast;
+                    tmem_ld1(dcol + 63, last);
+                    tmem_ld1(ucol, ulast);
+                    tmem_ld_wait();
+                    acc0.x = fmaf(__uint_as_float(last), __uint_as_float(ulast & 0xffff0000u), acc0.x);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_free[b]);
+                if (live) {
+                    const float o0 = (acc0.x + acc0.y) / den0, o1 = (acc1.x + acc1.y) / den1;
+                    if (i0 < T) {
+                        if (O32) ((float *)o)[seq_off + (long)i0 * D + e] = o0;
+                        else o[seq_off + (long)i0 * D + e] = __float2bfloat16_rn(o0);
+                    }
+                    if (i0 + 1 < T) {
+                        if (O32) ((float *)o)[seq_off + (long)(i0 + 1) * D + e] = o1;
+                        else o[seq_off + (long)(i0 + 1) * D + e] = __float2bfloat16_rn(o1);
+                    }
+                    if (e == 0) {
+                        if (i0 < T) {
+                            Lout[(long)bh * T + i0] = L0;
+                            lse[(long)bh * T + i0] = L0 + LN2 * log2f(den0);
+                        }
+                        if (i0 + 1 < T) {
+                            Lout[(long)bh * T + i0 + 1] = L1;
+                            lse[(long)bh * T + i0 + 1] = L1 + LN2 * log2f(den1);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == WS_CW0 + 4) {
+        // ================================================================== product warp
+        // The whole warp runs the loop convergently (the descriptors stay warp-uniform); one elected lane issues.
+        {
+            const uint32_t leader = elect_one();
+            ws_wait(&bar_om, 0, status, 16, abort);
+            const uint32_t idesc_1 = make_idesc_f16(128, MF, 0, 0, 0);        // fp16: X . OmegaT
+            const uint32_t idesc_p = make_idesc_f16(128, TC_C, 1, 0, 0);      // bf16: psi . chi'
+            const uint32_t idesc_2 = make_idesc_f16(128, 128, 1, 0, 0);       // bf16: MbT . psi, Vt . Pm
+            const uint64_t dom = make_smem_desc(smem_u32(smem + S::OFF_OM), 0, 1024, kSw128);
+            const int n_tiles = (n_end - n_begin) * NT;
+            int gq[2] = {0, 1};                            // next tile of each buffer
+            int step[2] = {0, 0};                          // 0: l, 1: P and the state part of Dt, 2: the intra-chunk part of Dt
+            int done_in_chunk[2] = {0, 0};                 // per image buffer: tiles whose last product has been issued
+            uint32_t spins = 0;
+            while ((gq[0] < n_tiles || gq[1] < n_tiles) && !*abort) {
+                bool progress = false;
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int g = gq[b];
+                    if (g >= n_tiles) continue;
+                    const uint32_t k = (uint32_t)g >> 1;
+                    const int c = g / NT;
+                    const uint32_t tl = tm + WS_L + b * 128;
+                    const uint32_t psi_a = smem_u32(smem + S::OFF_PSI + b * S::PSI_BYTES);
+                    const uint32_t img_a = smem_u32(smem + S::OFF_IMG + (c & 1) * G::IMG_CHUNK);
+                    if (step[b] == 0) {
+                        if (!mbar_test_wait(&bar_x[b], k & 1)) continue;
+                        if (k > 0 && !mbar_test_wait(&bar_free[b], (k - 1) & 1)) continue;
+                        tc_fence_after();
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks)
+                            mma_f16_ts_if(leader, tl, tm + WS_X + b * 64 + ks * 8, desc_adv(dom, (ks >> 2) * (MF * 128) + (ks & 3) * 32), idesc_1, ks > 0);
+                        tc_commit_if(leader, &bar_l[b]);
+                        step[b] = 1;
+                        progress = true;
+                    } else if (step[b] == 1) {
+                        if (!mbar_test_wait(&bar_psi[b], k & 1)) continue;
+                        if (!mbar_test_wait(&bar_img[c & 1], (c >> 1) & 1)) continue;
+                        tc_fence_after();
+                        const uint64_t dpsi = make_smem_desc(psi_a, 0, 1024, kSw128);
+                        const uint64_t dmb = make_smem_desc(img_a, 0, 1024, kSw128);
+                        const uint64_t dchi = make_smem_desc(img_a + G::IMG_M, 0, 1024, kSw128);
+#pragma unroll
+                        for (int ks = 0; ks < MF / 16; ++ks)
+                            mma_f16_ss_if(leader, tm + WS_P + b * 16, desc_adv(dpsi, (ks >> 2) * (128 * 128) + (ks & 3) * 32),
+                                          desc_adv(dchi, (ks >> 2) * (TC_C * 128) + (ks & 3) * 32), idesc_p, ks > 0);
+                        tc_commit_if(leader, &bar_p[b]);
+#pragma unroll
+                        for (int ks = 0; ks < MF / 16; ++ks) {
+                            const uint32_t koff = (ks >> 2) * (128 * 128) + (ks & 3) * 32;
+                            mma_f16_ss_if(leader, tl, desc_adv(dmb, koff), desc_adv(dpsi, koff), idesc_2, ks > 0);
+                        }
+                        step[b] = 2;
+                        progress = true;
+                    } else {
+                        if (!mbar_test_wait(&bar_pm[b], k & 1)) continue;
+                        tc_fence_after();
+                        const uint64_t ad = make_smem_desc(img_a + G::IMG_M + G::IMG_CHI, 0, 256, kSw32);
+                        const uint64_t bd = make_smem_desc(smem_u32(smem + S::OFF_PM + b * S::PM_BYTES), 0, 256, kSw32);
+                        mma_f16_ss_if(leader, tl, ad, bd, idesc_2, 1);
+                        tc_commit_if(leader, &bar_dt[b]);
+                        // the chunk's image is free once the last product of its eight tiles has completed
+                        if (++done_in_chunk[c & 1] == NT) {
+                            done_in_chunk[c & 1] = 0;
+                            tc_commit_if(leader, &bar_imgfree[c & 1]);
+                        }
+                        step[b] = 0;
+                        gq[b] = g + 2;
+                        progress = true;
+                    }
+                }
+                if (progress) spins = 0;
+                else if (++spins > kWaitLimit) {
+                    *abort = 1;
+                    if (status) atomicExch(status, 17);
+                }
+            }
+        }
+    } else if (warp == WS_CW0 + 5) {
+        // ================================================================== load warp
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&bar_om, G::IMG_OM);
+            bulk_g2s(smem + S::OFF_OM, om_img + (long)(om_per_head ? bh % H : 0) * G::IMG_OM, G::IMG_OM, &bar_om);
+            mbar_arrive_expect_tx(&bar_img[0], G::IMG_CHUNK);
+            bulk_g2s(smem + S::OFF_IMG, img_bh + (long)n_begin * G::IMG_CHUNK, G::IMG_CHUNK, &bar_img[0]);
+        }
+        auto r_piece = [&](int tok, int ch) -> uint4 {      // 8 elements of r[tok] as fp16 (exact for bf16 values in the fp16 range)
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (tok >= 0 && tok < T) val = *(const uint4 *)(r + seq_off + (long)tok * D + ch * 8);
+            else if (HIST && tok < 0 && tok >= -n_hist) val = *(const uint4 *)(hist_r + ((long)bh * n_hist + n_hist + tok) * D + ch * 8);
+            return make_uint4(bf2h_(val.x), bf2h_(val.y), bf2h_(val.z), bf2h_(val.w));
+        };
+        auto put_r = [&](int tok, int ch, uint4 v) {
+            const int rr = ring_row(tok);
+            *(uint4 *)(rwin + rr * S::ROWB + ((ch ^ (rr & 7)) << 4)) = v;
+        };
+        // the window before the first chunk: groups n_begin - 4 .. n_begin - 1
+        for (int idx = lane; idx < 4 * TC_C * CH; idx += 32) {
+            const int tok = (n_begin - 4) * TC_C + idx / CH, ch = idx % CH;
+            put_r(tok, ch, r_piece(tok, ch));
+        }
+        constexpr int PPL = TC_C * CH / 32;                 // 16-byte pieces of a 16-row group per lane
+        for (int n = n_begin; n < n_end; ++n) {
+            const int c = n - n_begin;
+            // chunk n's rows: r group n, q rows, boundary normaliser (loads first, then the wait for the buffers)
+            uint4 rp[PPL];
+#pragma unroll
+            for (int y = 0; y < PPL; ++y) {
+                const int idx = lane + 32 * y, tok = n * TC_C + idx / CH, ch = idx % CH;
+                rp[y] = r_piece(tok, ch);
+            }
+            float abv[MF / 32];
+#pragma unroll
+            for (int y = 0; y < MF / 32; ++y) abv[y] = ab_g[((long)bh * NC + n) * MF + lane + 32 * y];
+            // ring slot of group n held group n - 6, q / a_b buffer c & 1 held chunk n - 2: both last read in chunk n - 2
+            if (c >= 2) ws_wait(&bar_rowsfree[c & 1], ((c - 2) >> 1) & 1, status, 18, abort);
+#pragma unroll
+            for (int y = 0; y < PPL; ++y) {
+                const int idx = lane + 32 * y, rowi = idx / CH, ch = idx % CH;
+                put_r(n * TC_C + rowi, ch, rp[y]);
+            }
+#pragma unroll
+            for (int y = 0; y < PPL; ++y) {
+                const int idx = lane + 32 * y, rowi = idx / CH, ch = idx % CH, tok = n * TC_C + rowi;
+                uint4 val = make_uint4(0, 0, 0, 0);
+                if (tok < T) val = *(const uint4 *)(q + seq_off + (long)tok * D + ch * 8);
+                rp[y] = make_uint4(bf2h_(val.x), bf2h_(val.y), bf2h_(val.z), bf2h_(val.w));
+            }
+#pragma unroll
+            for (int y = 0; y < PPL; ++y) {
+                const int idx = lane + 32 * y, rowi = idx / CH, ch = idx % CH;
+                *(uint4 *)(smem + S::OFF_Q + (c & 1) * (TC_C * S::ROWB) + rowi * S::ROWB + (ch << 4)) = rp[y];
+            }
+#pragma unroll
+            for (int y = 0; y < MF / 32; ++y) ((float *)(smem + S::OFF_AB))[(c & 1) * MF + lane + 32 * y] = abv[y];
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&bar_rows[c & 1]);
+                // the next chunk's image, once the products of the chunk before this one have left its buffer
+                if (n + 1 < n_end) {
+                    if (c >= 1) ws_wait(&bar_imgfree[(c + 1) & 1], ((c - 1) >> 1) & 1, status, 19, abort);
+                    mbar_arrive_expect_tx(&bar_img[(c + 1) & 1], G::IMG_CHUNK);
+                    bulk_g2s(smem + S::OFF_IMG + ((c + 1) & 1) * G::IMG_CHUNK, img_bh + (long)(n + 1) * G::IMG_CHUNK, G::IMG_CHUNK,
+                             &bar_img[(c + 1) & 1]);
+                }
+            }
+            __syncwarp();
+        }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem_base_s, 512);
+    __syncwarp();
+    if (warp == WS_CW0 + 4) tmem_dealloc(tmem_base_s, 512);
 }
 
 // ------------------------------------------------------------------ host side
@@ -855,7 +1071,7 @@ template <int D, int MF>
 static int fwd_tc_impl(const TcArgs &a, cudaStream_t st)
 {
     using G = TcGeom<D, MF>;
-    using S = FwdTcSmem<D, MF>;
+    using S = FwdWsSmem<D, MF>;
     const int NC = (a.T + TC_C - 1) / TC_C, BH = a.B * a.H;
     LaunchScope sc = {st, 0};
     const int n_om = a.omega_stride ? a.H : 1;
@@ -893,7 +1109,7 @@ static int fwd_tc_impl(const TcArgs &a, cudaStream_t st)
     const int cpc = a.chunks_per_cta;
     auto launch = [&](auto kern) {
         sc.check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        LS_LAUNCH(sc, "fwd_tc", kern<<<dim3((NC + cpc - 1) / cpc, BH), TC_NT, smem, st>>>(
+        LS_LAUNCH(sc, "fwd_tc", kern<<<dim3((NC + cpc - 1) / cpc, BH), WS_NT, smem, st>>>(
             (const bf16 *)a.q, (const bf16 *)a.r, (const bf16 *)a.u, a.om_img, a.omega_stride != 0, a.H, a.T, a.W, NC, cpc,
             a.log2_eps_m, a.images, a.ab, a.o32 ? (bf16 *)a.o32 : (bf16 *)a.o, a.L, a.lse, a.status, a.m_real,
             (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist));
