@@ -141,7 +141,7 @@ int linsimp_fwd(const linsimp_params *p,
  *        the n_hist tokens before the segment, oldest first; they act only as anchors.
  * Outputs cover the segment's T tokens.  Available where the tensor-core forward is
  * (bf16 I/O, default algo, d in {64,128}, m in {32,64,128}); LINSIMP_EUNSUPPORTED otherwise.
- * There is no backward for a continued segment.
+ * Its backward is linsimp_bwd_continue.
  */
 int linsimp_fwd_continue(const linsimp_params *p,
                          const void *q, const void *k, const void *v, const void *r, const void *u,
@@ -150,6 +150,39 @@ int linsimp_fwd_continue(const linsimp_params *p,
                          const void *hist_r, const void *hist_u, int32_t n_hist,
                          void *o, float *rowmax_L, float *lse,
                          float *S_final, float *z_final,
+                         void *workspace, size_t workspace_bytes, linsimp_stream stream);
+
+/*
+ * Backward of a continued segment (Theorem 1 read backwards: the only paths between a segment
+ * and the rest of the sequence are the state M, a it starts from and ends with and the W-1
+ * anchor rows before it; App. C for the sweeps themselves).  For a loss
+ *     sum(dO * o_segment) + f(S_final, z_final)
+ * with dS_final = df/dS_final and dz_final = df/dz_final known, it returns the gradients with
+ * respect to the segment's own q, k, v, r, u, to the history anchors and to the state the
+ * segment started from.  Chunked training over a long sequence walks the segments last to
+ * first: dS_init, dz_init of one call are dS_final, dz_final of the call for the segment
+ * before, and d_hist_r, d_hist_u are added by the caller to dr, du of the last n_hist rows
+ * before the segment (the rows hist_r, hist_u were copied from).
+ *   in : q,k,v,r,u [B,H,T,d], omega, S_init, z_init, hist_r, hist_u, n_hist as in
+ *        linsimp_fwd_continue; rowmax_L, lse [B,H,T] from that call; dO [B,H,T,d];
+ *        dS_final [B,H,m,d], dz_final [B,H,m] fp32 (both or neither null: null = zero)
+ *   out: dq,dk,dv,dr,du [B,H,T,d] io_dtype (overwritten);
+ *        d_hist_r, d_hist_u [B,H,n_hist,d] io_dtype (overwritten; null when n_hist = 0);
+ *        dS_init [B,H,m,d], dz_init [B,H,m] fp32 (both or neither null), in the convention of
+ *        the state tensors (gradient with respect to those very numbers)
+ *   workspace: linsimp_workspace_bytes(p, LINSIMP_OP_BWD).  LINSIMP_FLAG_REUSE_FWD_STATE is not
+ *        accepted here (LINSIMP_EINVAL): the segment's pre-pass always runs.
+ * Available where linsimp_fwd_continue is; LINSIMP_EUNSUPPORTED otherwise.
+ */
+int linsimp_bwd_continue(const linsimp_params *p,
+                         const void *q, const void *k, const void *v, const void *r, const void *u,
+                         const float *omega,
+                         const float *S_init, const float *z_init,
+                         const void *hist_r, const void *hist_u, int32_t n_hist,
+                         const float *rowmax_L, const float *lse, const void *dO,
+                         const float *dS_final, const float *dz_final,
+                         void *dq, void *dk, void *dv, void *dr, void *du,
+                         void *d_hist_r, void *d_hist_u, float *dS_init, float *dz_init,
                          void *workspace, size_t workspace_bytes, linsimp_stream stream);
 
 /*

@@ -34,7 +34,8 @@ typedef struct linsimp_umma_probe {
  * build are accepted (kind::f16, fp32 accumulator, fp16 or bf16 for both operands, M = 128,
  * N a multiple of 16 up to 256, 32/64/128-byte swizzle, K steps inside the image); anything
  * else returns -2 before a launch.  -1: null pointer or size out of range; -5: CUDA error.
- * `status` (device int, nullable) receives code 1 if the kernel's wait on the product gives up.
+ * `status` (two device ints, nullable): [0] receives code 1 if the kernel's wait on the product gives up, [1] the
+ * clock ticks from the first issue to the completion of the chain.
  */
 int linsimp_debug_umma(const void *a_img, const void *b_img, const linsimp_umma_probe *probe, float *out,
                        int *status, void *stream);

@@ -19,7 +19,7 @@ EXPORTS = ("linsimp_workspace_bytes", "linsimp_fwd", "linsimp_bwd", "linsimp_dec
            "linsimp_strerror", "linsimp_version", "linsimp_last_launch_count",
            "linsimp_profile_enable", "linsimp_profile_read", "linsimp_read_status", "linsimp_fwd_static",
            "linsimp_qkr_normalize", "linsimp_qkr_normalize_bwd", "linsimp_gate_rmsnorm", "linsimp_gate_rmsnorm_bwd",
-           "linsimp_fwd_padded", "linsimp_bwd_padded", "linsimp_ring_fill_padded")
+           "linsimp_fwd_padded", "linsimp_bwd_padded", "linsimp_ring_fill_padded", "linsimp_bwd_continue")
 
 
 class LinSimpError(RuntimeError):
@@ -62,6 +62,9 @@ def load_library():
     lib.linsimp_fwd_continue.restype = ctypes.c_int
     lib.linsimp_fwd_continue.argtypes = [pp, vp, vp, vp, vp, vp, fp, fp, fp, vp, vp, ctypes.c_int32, vp, fp, fp, fp, fp,
                                          vp, ctypes.c_size_t, vp]
+    lib.linsimp_bwd_continue.restype = ctypes.c_int
+    lib.linsimp_bwd_continue.argtypes = [pp, vp, vp, vp, vp, vp, fp, fp, fp, vp, vp, ctypes.c_int32, fp, fp, vp, fp, fp,
+                                         vp, vp, vp, vp, vp, vp, vp, fp, fp, vp, ctypes.c_size_t, vp]
     lib.linsimp_ring_fill.restype = ctypes.c_int
     lib.linsimp_ring_fill.argtypes = [pp, vp, vp, ctypes.c_int64, vp, vp, vp]
     lib.linsimp_decode_prepare.restype = ctypes.c_int
@@ -214,6 +217,45 @@ def fwd_continue(q, k, v, r, u, omega, state=None, history=None, W=64, eps=1e-30
     if return_state:
         return o, L, lse, S, z
     return o, L, lse
+
+
+def bwd_continue(q, k, v, r, u, omega, L, lse, dO, state=None, history=None, d_state=None, W=64, eps=1e-30,
+                 workspace=None, stream=None):
+    """linsimp_bwd_continue: backward of a segment run with fwd_continue.
+
+    state = (S_init, z_init) or None, history = (hist_r, hist_u) or None as given to fwd_continue;
+    d_state = (dS_final, dz_final) or None: the gradient later segments send into the state after this one.
+    Returns (dq, dk, dv, dr, du), (d_hist_r, d_hist_u) or None, (dS_init, dz_init)."""
+    lib = load_library()
+    _dev(q, k, v, r, u, omega, L, lse, dO)
+    B, H, T, d = q.shape
+    m = omega.shape[-1]
+    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, ALGO_DEFAULT, eps)
+    S0 = z0 = hr = hu = dSf = dzf = None
+    n_hist = 0
+    if state is not None:
+        S0, z0 = state
+        _dev(S0, z0)
+    if history is not None and history[0].shape[2] > 0:
+        hr, hu = history
+        _dev(hr, hu)
+        n_hist = hr.shape[2]
+    if d_state is not None:
+        dSf, dzf = d_state
+        _dev(dSf, dzf)
+    grads = [torch.empty_like(q) for _ in range(5)]
+    dh = None
+    if n_hist:
+        dh = (torch.empty_like(hr), torch.empty_like(hu))
+    dS0 = torch.empty((B, H, m, d), dtype=torch.float32, device=q.device)
+    dz0 = torch.empty((B, H, m), dtype=torch.float32, device=q.device)
+    ws, ws_bytes = _workspace(p, OP_BWD, workspace, q.device)
+    _check(lib.linsimp_bwd_continue(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),
+                                    _ptr(S0), _ptr(z0), _ptr(hr), _ptr(hu), n_hist, _ptr(L), _ptr(lse), _ptr(dO),
+                                    _ptr(dSf), _ptr(dzf), *[_ptr(g) for g in grads],
+                                    _ptr(dh[0]) if dh else None, _ptr(dh[1]) if dh else None, _ptr(dS0), _ptr(dz0),
+                                    _ptr(ws), ws_bytes, _stream(stream)))
+    return tuple(grads), dh, (dS0, dz0)
 
 
 def ring_fill(r, u, ring_r, ring_u, t_first=0, stream=None):

@@ -154,7 +154,8 @@ bool use_tc(const linsimp_params *p, int op)
 }
 
 struct TcLayout {
-    size_t status, chi_ml, segtot, images, ab, om_img, chi32, gstates, segsum, dv_intra, dchi_intra, dr_acc, du_acc, total;
+    size_t status, chi_ml, segtot, images, ab, om_img, chi32, gstates, segsum, dv_intra, dchi_intra, dr_acc, du_acc, dhr_acc,
+        dhu_acc, total;
 };
 
 // feature rank the tensor-core kernels run with: ranks below 64 are zero-padded to 64
@@ -196,6 +197,11 @@ TcLayout tc_layout(const linsimp_params *p, int op)
         off = align_up(off + BH * p->T * p->d * sizeof(float), 1024);
         L.du_acc = off;
         off = align_up(off + BH * p->T * p->d * sizeof(float), 1024);
+        // a continued segment: gradients of up to W - 1 <= 63 history anchors per unit
+        L.dhr_acc = off;
+        off = align_up(off + BH * 64 * p->d * sizeof(float), 1024);
+        L.dhu_acc = off;
+        off = align_up(off + BH * 64 * p->d * sizeof(float), 1024);
     }
     L.total = off;
     return L;
@@ -292,10 +298,20 @@ int run_tc(const linsimp_params *p, const void *q, const void *k, const void *v,
     return finish(op, tc_fwd_run(a, (cudaStream_t)stream));
 }
 
+// what a continued segment adds to the backward's arguments
+struct TcBwdHistory {
+    const float *S_init = nullptr, *z_init = nullptr;
+    const void *hist_r = nullptr, *hist_u = nullptr;
+    int n_hist = 0;
+    const float *dS_final = nullptr, *dz_final = nullptr;
+    float *dS_init = nullptr, *dz_init = nullptr;
+    void *d_hist_r = nullptr, *d_hist_u = nullptr;
+};
+
 int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
                const float *omega, const void *o, const float *rowmax_L, const float *lse, const void *dO, void *dq, void *dk,
                void *dv, void *dr, void *du, void *workspace, size_t workspace_bytes, linsimp_stream stream,
-               const int *seq_lens)
+               const int *seq_lens, const TcBwdHistory &hist = TcBwdHistory())
 {
     const TcLayout TL = tc_layout(p, LINSIMP_OP_BWD);
     if (!workspace || workspace_bytes < TL.total) return LINSIMP_EWORKSPACE;
@@ -325,6 +341,11 @@ int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void
     a.dchi_intra = (float *)(tws + TL.dchi_intra);
     a.dr_acc = (float *)(tws + TL.dr_acc);
     a.du_acc = (float *)(tws + TL.du_acc);
+    a.dhr_acc = (float *)(tws + TL.dhr_acc);
+    a.dhu_acc = (float *)(tws + TL.dhu_acc);
+    a.S_init = hist.S_init; a.z_init = hist.z_init; a.hist_r = hist.hist_r; a.hist_u = hist.hist_u; a.n_hist = hist.n_hist;
+    a.dS_final = hist.dS_final; a.dz_final = hist.dz_final; a.dS_init = hist.dS_init; a.dz_init = hist.dz_init;
+    a.d_hist_r = hist.d_hist_r; a.d_hist_u = hist.d_hist_u;
     if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
     return finish(LINSIMP_OP_BWD, tc_bwd_run(a, (cudaStream_t)stream));
 }
@@ -448,6 +469,33 @@ int linsimp_fwd_continue(const linsimp_params *p, const void *q, const void *k, 
     TcHistory h;
     h.S_init = S_init; h.z_init = z_init; h.hist_r = hist_r; h.hist_u = hist_u; h.n_hist = n_hist;
     return run_tc(p, q, k, v, r, u, omega, o, rowmax_L, lse, S_final, z_final, workspace, workspace_bytes, stream, 0, h);
+}
+
+int linsimp_bwd_continue(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                         const float *omega, const float *S_init, const float *z_init, const void *hist_r,
+                         const void *hist_u, int32_t n_hist, const float *rowmax_L, const float *lse, const void *dO,
+                         const float *dS_final, const float *dz_final, void *dq, void *dk, void *dv, void *dr, void *du,
+                         void *d_hist_r, void *d_hist_u, float *dS_init, float *dz_init, void *workspace,
+                         size_t workspace_bytes, linsimp_stream stream)
+{
+    if (!params_ok(p, LINSIMP_OP_BWD)) return LINSIMP_EINVAL;
+    if (!q || !k || !v || !r || !u || !omega || !rowmax_L || !lse || !dO || !dq || !dk || !dv || !dr || !du) return LINSIMP_EINVAL;
+    if ((S_init == nullptr) != (z_init == nullptr) || (dS_final == nullptr) != (dz_final == nullptr) ||
+        (dS_init == nullptr) != (dz_init == nullptr))
+        return LINSIMP_EINVAL;
+    if (n_hist < 0 || n_hist > p->W - 1 || (n_hist > 0 && (!hist_r || !hist_u || !d_hist_r || !d_hist_u))) return LINSIMP_EINVAL;
+    if (p->flags & LINSIMP_FLAG_REUSE_FWD_STATE) return LINSIMP_EINVAL;      // the segment's pre-pass always runs
+    if (!shape_supported(p) || !use_tc(p, LINSIMP_OP_BWD)) return LINSIMP_EUNSUPPORTED;
+    const void *ptrs[] = {q, k, v, r, u, omega, dO, dq, dk, dv, dr, du, S_init, z_init, hist_r, hist_u, dS_final, dz_final,
+                          d_hist_r, d_hist_u, dS_init, dz_init};
+    for (const void *x : ptrs)
+        if (x && !aligned16(x)) return LINSIMP_EALIGN;
+    TcBwdHistory h;
+    h.S_init = S_init; h.z_init = z_init; h.hist_r = hist_r; h.hist_u = hist_u; h.n_hist = n_hist;
+    h.dS_final = dS_final; h.dz_final = dz_final; h.dS_init = dS_init; h.dz_init = dz_init;
+    h.d_hist_r = d_hist_r; h.d_hist_u = d_hist_u;
+    return run_tc_bwd(p, q, k, v, r, u, omega, nullptr, rowmax_L, lse, dO, dq, dk, dv, dr, du, workspace, workspace_bytes, stream,
+                      nullptr, h);
 }
 
 int linsimp_ring_fill(const linsimp_params *p, const void *r, const void *u, int64_t t_first, void *ring_r, void *ring_u,

@@ -105,6 +105,9 @@ __device__ __forceinline__ int anchor_of(int i, int x) { return i - ((i - x) & 6
 // pass per block in DOT mode computes only that (the tile pipeline up to dpsiN, no gradients) and adds it to
 // delta[bh][i]; the second pass per block in EXT mode takes the total from there and writes fp32 gradients that are
 // summed over the blocks.
+// MODE 3 (HIST) is the backward of a segment that continues a sequence: the anchors of the n_hist tokens before the
+// segment come from hist_r, hist_u, and what the segment's queries contribute to the gradients of those anchors
+// leaves through the accumulators dhr_acc, dhu_acc [BH][n_hist][D].
 template <int D, int MF, int MODE>
 __global__ void __launch_bounds__(BNT, 1)
 k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__restrict__ u,
@@ -113,9 +116,12 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
          const uint8_t *__restrict__ images, const float *__restrict__ ab_g, bf16 *__restrict__ dq,
          float *__restrict__ dr_acc, float *__restrict__ du_acc, float *__restrict__ gstates,
          float *__restrict__ dv_intra, float *__restrict__ dchi_intra, int *__restrict__ status,
-         const float *__restrict__ delta_ext, int grad32, float *__restrict__ delta_out, const int *__restrict__ seq_lens)
+         const float *__restrict__ delta_ext, int grad32, float *__restrict__ delta_out, const int *__restrict__ seq_lens,
+         const bf16 *__restrict__ hist_r, const bf16 *__restrict__ hist_u, int n_hist_arg, float *__restrict__ dhr_acc,
+         float *__restrict__ dhu_acc)
 {
-    constexpr bool EXT = MODE == 1, DOT = MODE == 2;
+    constexpr bool EXT = MODE == 1, DOT = MODE == 2, HIST = MODE == 3;
+    const int n_hist = HIST ? n_hist_arg : 0;
     using S = BwdTcSmem<D, MF>;
     constexpr int CPT = MF / BR;                      // feature columns per thread in the row passes
     constexpr float LOG2E = 1.4426950408889634f;
@@ -254,6 +260,9 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 if (tok >= 0 && tok < T) {
                     rv = *(const uint4 *)(r + seq_off + (long)tok * D + ch * 8);
                     uv = *(const uint4 *)(u + seq_off + (long)tok * D + ch * 8);
+                } else if (HIST && tok < 0 && tok >= -n_hist) {      // anchors from before the segment
+                    rv = *(const uint4 *)(hist_r + ((long)bh * n_hist + n_hist + tok) * D + ch * 8);
+                    uv = *(const uint4 *)(hist_u + ((long)bh * n_hist + n_hist + tok) * D + ch * 8);
                 }
                 const int rr = ring_row(tok);
                 // r is kept as fp16 (exact for bf16 values in the fp16 range): X = q * r is then one packed multiply
@@ -346,7 +355,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
             const int slot = t & 63;
             const int c = anchor_of(i, slot);
             const int s = i - c;
-            const bool valid = (s < W) && (c >= 0) && (i < T);
+            const bool valid = (s < W) && (c >= -n_hist) && (i < T);
             const int wrow = ring_row(c);                 // always inside the window (rows outside [0,T) hold zeros)
             if (tile == 0) {
                 phase1(0);
@@ -533,8 +542,14 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     if (k0 <= 15) {
                         // k0 = 2 * tile + qi here (the group that takes the chunk's own tokens in): a switch over the tile
                         // makes the slot a compile-time register index
-                        float *dst = du_acc + seq_off + (long)(iq - 64) * D + t;
-                        const bool live = iq - 64 >= 0 && iq < T + 64;
+                        // the anchor that leaves is token iq - 64: inside the segment, among its history rows, or nowhere
+                        const int ca = iq - 64;
+                        float *dst = du_acc + seq_off + (long)ca * D + t;
+                        bool live = ca >= 0 && ca < T;
+                        if (HIST && ca < 0 && ca >= -n_hist) {
+                            dst = dhu_acc + ((long)bh * n_hist + n_hist + ca) * D + t;
+                            live = true;
+                        }
 #define LS_FLUSH_DU(X) { if (live) atomicAdd(dst, __uint_as_float(wv[X])); wv[X] = 0u; }
                         switch (tile) {
                         case 0: LS_FLUSH_DU(0 + qi) break;
@@ -723,8 +738,13 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     } else {
                         // anchor iq takes residue k0 = 2 * tile + qi over: what the slot holds leaves first (a switch over
                         // the tile makes it a compile-time register index)
-                        float *dst = dr_acc + seq_off + (long)(iq - 64) * D + t;
-                        const bool live = iq - 64 >= 0 && iq < T + 64;
+                        const int ca = iq - 64;
+                        float *dst = dr_acc + seq_off + (long)ca * D + t;
+                        bool live = ca >= 0 && ca < T;
+                        if (HIST && ca < 0 && ca >= -n_hist) {
+                            dst = dhr_acc + ((long)bh * n_hist + n_hist + ca) * D + t;
+                            live = true;
+                        }
 #define LS_FLUSH_DR(X) { if (live) atomicAdd(dst, __uint_as_float(wv[X])); wv[X] = 0u; }
                         switch (tile) {
                         case 0: LS_FLUSH_DR(0 + qi) break;
@@ -836,6 +856,9 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
             if (ca >= 0 && ca < T) {
                 atomicAdd(du_acc + seq_off + (long)ca * D + t, __uint_as_float(wu[x]));
                 atomicAdd(dr_acc + seq_off + (long)ca * D + t, __uint_as_float(wr_[x]));
+            } else if (HIST && ca < 0 && ca >= -n_hist) {
+                atomicAdd(dhu_acc + ((long)bh * n_hist + n_hist + ca) * D + t, __uint_as_float(wu[x]));
+                atomicAdd(dhr_acc + ((long)bh * n_hist + n_hist + ca) * D + t, __uint_as_float(wr_[x]));
             }
         }
     }
@@ -939,7 +962,8 @@ template <int D, int MF>
 __global__ void __launch_bounds__(256, 2)
 k_bwd_kv_tc(const bf16 *__restrict__ v, int T, int NC, const float *__restrict__ gstates, const float *__restrict__ segsum,
             const float *__restrict__ dv_intra, const float *__restrict__ dchi_intra, float *__restrict__ chi_dl,
-            bf16 *__restrict__ dv, int grad32, int seg_len)
+            bf16 *__restrict__ dv, int grad32, int seg_len, const float *__restrict__ dS_fin, const float *__restrict__ dz_fin,
+            int state_m, int m_real)
 {
     constexpr int LDD = D + 4, LDK = D + 4, LDC = MF + 4;
     extern __shared__ float sm[];
@@ -957,11 +981,14 @@ k_bwd_kv_tc(const bf16 *__restrict__ v, int T, int NC, const float *__restrict__
         for (int s2 = seg + 1; s2 < NSEG; ++s2) acc += segsum[((long)bh * NSEG + s2) * E + idx];
         const int p = idx / D, e0 = idx - p * D;
         const int e = (((e0 >> 2) ^ (p & 7)) << 2) | (e0 & 3);         // the tile kernel permutes the 16-byte pieces of a row
+        // (a continued segment: the gradient that later segments send into the state after this one)
+        if (dS_fin && p < m_real) acc += dS_fin[((long)bh * state_m + p) * D + e];
         Ds[p * LDD + e] = acc;
     }
     for (int p = threadIdx.x; p < MF; p += 256) {
         float acc = 0.f;
         for (int s2 = seg + 1; s2 < NSEG; ++s2) acc += segsum[((long)bh * NSEG + s2) * E + (long)MF * D + p];
+        if (dz_fin && p < m_real) acc += dz_fin[(long)bh * state_m + p];
         es[p] = acc;
     }
     const int n_hi = min(NC, (seg + 1) * seg_len) - 1;
@@ -1088,7 +1115,8 @@ struct Kv5Smem {
 __global__ void __launch_bounds__(256, 2)
 k_bwd_kv_tc5(const bf16 *__restrict__ v, int T, int NC, const float *__restrict__ gstates, const float *__restrict__ segsum,
              const float *__restrict__ dv_intra, const float *__restrict__ dchi_intra, float *__restrict__ chi_dl,
-             bf16 *__restrict__ dv, int seg_len, int *__restrict__ status)
+             bf16 *__restrict__ dv, int seg_len, int *__restrict__ status, const float *__restrict__ dS_fin,
+             const float *__restrict__ dz_fin)
 {
     constexpr int D = 128, MF = 128, NX = MF * D / 4 / 256;    // 16 float4 of D per thread
     using S = Kv5Smem;
@@ -1118,11 +1146,18 @@ k_bwd_kv_tc5(const bf16 *__restrict__ v, int T, int NC, const float *__restrict_
             const float4 w = ((const float4 *)(segsum + ((long)bh * NSEG + s2) * E))[tid + 256 * x];
             acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
         }
+        if (dS_fin) {
+            // a continued segment: the gradient that later segments send into the state after this one ([p][e], plain order)
+            const int p = warp + 8 * x, e = (lane ^ (p & 7)) * 4;
+            const float4 w = *(const float4 *)(dS_fin + ((long)bh * MF + p) * D + e);
+            acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
+        }
         Dr[x] = acc;
     }
     const int row = (warp & 3) * 32 + lane, half = warp >> 2;   // accumulator row (p resp. e) and token half of the epilogues
     float es = 0.f;                                             // e[p] for p = row
     for (int s2 = seg + 1; s2 < NSEG; ++s2) es += segsum[((long)bh * NSEG + s2) * E + (long)MF * D + row];
+    if (dz_fin) es += dz_fin[(long)bh * MF + row];
     auto store_images = [&]() {
 #pragma unroll
         for (int x = 0; x < NX; ++x) {
@@ -1543,6 +1578,29 @@ k_bwd_dk_tc5(const bf16 *__restrict__ k, const float *__restrict__ omega, long o
     if (warp == 0) tmem_dealloc(tmem_base_s, 128);
 }
 
+// Gradient with respect to the state a continued segment started from: every chunk's state gradient plus what flows into
+// the state after the segment.  dS_init [BH][state_m][D] (plain [p][e] order), dz_init [BH][state_m].  grid (BH).
+__global__ void __launch_bounds__(256) k_state_grad_total(const float *__restrict__ segsum, int NSEG, int MF, int D, int m_real,
+                                                          int state_m, const float *__restrict__ dS_fin,
+                                                          const float *__restrict__ dz_fin, float *__restrict__ dS_init,
+                                                          float *__restrict__ dz_init)
+{
+    const int bh = blockIdx.x;
+    const long E = (long)MF * D + MF;
+    for (int idx = threadIdx.x; idx < m_real * D; idx += 256) {
+        const int p = idx / D, e = idx - p * D;
+        const int e0 = (((e >> 2) ^ (p & 7)) << 2) | (e & 3);          // where the tile kernel's permuted rows keep channel e
+        float acc = dS_fin ? dS_fin[((long)bh * state_m + p) * D + e] : 0.f;
+        for (int s2 = 0; s2 < NSEG; ++s2) acc += segsum[((long)bh * NSEG + s2) * E + (long)p * D + e0];
+        dS_init[((long)bh * state_m + p) * D + e] = acc;
+    }
+    for (int p = threadIdx.x; p < m_real; p += 256) {
+        float acc = dz_fin ? dz_fin[(long)bh * state_m + p] : 0.f;
+        for (int s2 = 0; s2 < NSEG; ++s2) acc += segsum[((long)bh * NSEG + s2) * E + (long)MF * D + p];
+        dz_init[(long)bh * state_m + p] = acc;
+    }
+}
+
 // n is a multiple of 8 (d is 64 or 128) and both buffers are 16-byte aligned
 __global__ void k_f32_to_bf16(const float *__restrict__ src, bf16 *__restrict__ dst, long n)
 {
@@ -1577,6 +1635,11 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
         sc.check(cudaMemsetAsync(a.dr_acc, 0, sizeof(float) * ntok, st));
         sc.check(cudaMemsetAsync(a.du_acc, 0, sizeof(float) * ntok, st));
     }
+    const long nhist = (long)BH * a.n_hist * D;
+    if (a.n_hist > 0) {
+        sc.check(cudaMemsetAsync(a.dhr_acc, 0, sizeof(float) * nhist, st));
+        sc.check(cudaMemsetAsync(a.dhu_acc, 0, sizeof(float) * nhist, st));
+    }
     const int smem = S::TOTAL + 1024;
     const int cpc = a.chunks_per_cta;
     auto launch = [&](auto kern) {
@@ -1584,13 +1647,15 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
         LS_LAUNCH(sc, "bwd_tc", kern<<<dim3((NC + cpc - 1) / cpc, BH), BNT, smem, st>>>(
             (const bf16 *)a.q, (const bf16 *)a.r, (const bf16 *)a.u, (const bf16 *)a.dO, a.L, a.lse,
             a.om_img, a.omega_stride != 0, a.H, a.T, a.W, NC, cpc, a.images, a.ab, (bf16 *)a.dq, a.dr_acc, a.du_acc,
-            a.gstates, a.dv_intra, a.dchi_intra, a.status, a.delta_ext, a.grad32, a.delta_out, a.seq_lens));
+            a.gstates, a.dv_intra, a.dchi_intra, a.status, a.delta_ext, a.grad32, a.delta_out, a.seq_lens,
+            (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist, a.dhr_acc, a.dhu_acc));
     };
     if (a.delta_out) {
         launch(k_bwd_tc<D, MF, 2>);
         return sc.result();                   // first pass of a feature block: only its part of the layer's dO . o
     }
     if (a.delta_ext) launch(k_bwd_tc<D, MF, 1>);
+    else if (a.n_hist > 0) launch(k_bwd_tc<D, MF, 3>);
     else launch(k_bwd_tc<D, MF, 0>);
     // Segments of the key/value sweep: one wave of CTAs (two per SM) where the sequence is long enough, never shorter
     // than KV_SEG chunks (the workspace holds one partial sum per KV_SEG chunks).
@@ -1605,11 +1670,16 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
     if (D == 128 && MF == 128 && !a.grad32) {
         sc.check(cudaFuncSetAttribute(k_bwd_kv_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, Kv5Smem::TOTAL + 1024));
         LS_LAUNCH(sc, "bwd_kv_tc", k_bwd_kv_tc5<<<dim3(NSEG, BH), 256, Kv5Smem::TOTAL + 1024, st>>>(
-            (const bf16 *)a.v, a.T, NC, a.gstates, a.segsum, a.dv_intra, a.dchi_intra, a.chi32, (bf16 *)a.dv, seg_len, a.status));
+            (const bf16 *)a.v, a.T, NC, a.gstates, a.segsum, a.dv_intra, a.dchi_intra, a.chi32, (bf16 *)a.dv, seg_len, a.status,
+            a.dS_final, a.dz_final));
     } else {
         LS_LAUNCH(sc, "bwd_kv_tc", k_bwd_kv_tc<D, MF><<<dim3(NSEG, BH), 256, kv_smem, st>>>(
-            (const bf16 *)a.v, a.T, NC, a.gstates, a.segsum, a.dv_intra, a.dchi_intra, a.chi32, (bf16 *)a.dv, a.grad32, seg_len));
+            (const bf16 *)a.v, a.T, NC, a.gstates, a.segsum, a.dv_intra, a.dchi_intra, a.chi32, (bf16 *)a.dv, a.grad32, seg_len,
+            a.dS_final, a.dz_final, a.state_m, a.m_real));
     }
+    if (a.dS_init)
+        LS_LAUNCH(sc, "state_grad_total", k_state_grad_total<<<BH, 256, 0, st>>>(a.segsum, NSEG, MF, D, a.m_real, a.state_m, a.dS_final,
+                                                                             a.dz_final, a.dS_init, a.dz_init));
     const int dk_smem = sizeof(float) * (D * (MF + 4) + BC * (D + 4) + BC * (MF + 4) + BC);
     sc.check(cudaFuncSetAttribute(k_bwd_dk_tc<D, MF>, cudaFuncAttributeMaxDynamicSharedMemorySize, dk_smem));
     if (a.grad32) {
@@ -1625,6 +1695,10 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
     if (!a.hold_acc) {
         LS_LAUNCH(sc, "convert_out", k_f32_to_bf16<<<2368, 256, 0, st>>>(a.dr_acc, (bf16 *)a.dr, ntok));
         LS_LAUNCH(sc, "convert_out", k_f32_to_bf16<<<2368, 256, 0, st>>>(a.du_acc, (bf16 *)a.du, ntok));
+    }
+    if (a.n_hist > 0) {
+        LS_LAUNCH(sc, "convert_out", k_f32_to_bf16<<<64, 256, 0, st>>>(a.dhr_acc, (bf16 *)a.d_hist_r, nhist));
+        LS_LAUNCH(sc, "convert_out", k_f32_to_bf16<<<64, 256, 0, st>>>(a.dhu_acc, (bf16 *)a.d_hist_u, nhist));
     }
     return sc.result();
 }

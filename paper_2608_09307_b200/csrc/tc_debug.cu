@@ -54,7 +54,9 @@ __global__ void __launch_bounds__(128) k_umma_probe(const uint4 *__restrict__ a_
         __syncthreads();
         tc_fence_after();
     }
+    long long t_issue = 0;
     if (threadIdx.x == 0) {
+        t_issue = clock64();
         for (int k = 0; k < pr.nk; ++k) {
             const uint64_t bd = make_smem_desc(smem_u32(b_s) + pr.b_koff[k], pr.b_lbo, pr.b_sbo, pr.b_layout);
             if (pr.a_from_tmem) {
@@ -67,6 +69,8 @@ __global__ void __launch_bounds__(128) k_umma_probe(const uint4 *__restrict__ a_
         tc_commit(&bar);
     }
     mbar_wait(&bar, 0, status, 1);
+    // clock ticks from the first issue to the completion of the chain as thread 0 sees it (second word of `status`)
+    if (threadIdx.x == 0 && status) status[1] = (int)(clock64() - t_issue);
     tc_fence_after();
     for (int c0 = 0; c0 < pr.n_out; c0 += 16) {
         uint32_t r[16];

@@ -51,6 +51,11 @@ struct TcArgs {
     float *dv_intra;                 // [BH][NC][16][d]  intra-chunk part of dv
     float *dchi_intra;               // [BH][NC][16][m]  intra-chunk part of d chi'
     float *dr_acc, *du_acc;          // [BH][T][d] fp32 accumulators of the anchor gradients
+    // backward of a continued segment (all nullable / 0 otherwise; S_init, z_init, hist_r, hist_u, n_hist as in the forward)
+    const float *dS_final, *dz_final;   // gradient flowing into the state after the segment ([BH][state_m][d], [BH][state_m])
+    float *dS_init, *dz_init;           // out: gradient with respect to the state the segment started from
+    void *d_hist_r, *d_hist_u;          // out: [BH][n_hist][d] gradient with respect to the history anchors
+    float *dhr_acc, *dhu_acc;           // [BH][n_hist][d] fp32 accumulators behind them
 };
 
 int tc_supported(int d, int m);

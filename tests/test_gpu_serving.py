@@ -48,6 +48,92 @@ def test_chunked_prefill_equals_one_forward(d, m, W, cuts):
     assert np.abs(to64(torch.cat(lses, dim=2)).reshape(B * H, T) - lse_ref).max() < 5e-2
 
 
+@pytest.mark.parametrize("d,m,W,cuts", [(128, 128, 64, (137, 300)), (64, 128, 64, (16, 77, 200)), (64, 32, 33, (5, 90)),
+                                        (128, 64, 64, (1, 2, 150)), (64, 64, 7, (40, 41, 130)), (128, 128, 64, (2100, 4300))])
+def test_chunked_backward_equals_one_backward(d, m, W, cuts):
+    """Chunked training: the forward runs segment by segment (linsimp_fwd_continue), the backward walks the segments
+    last to first (linsimp_bwd_continue), handing the state gradient and the gradients of the W-1 history anchors
+    from each segment to the one before.  The result must be the gradient of the whole sequence, which the oracle
+    computes in one piece.  Cut points inside a window, segments of one token and segmented state walks included."""
+    B, H, T = 1, 2, cuts[-1]
+    t = synth.make_inputs(B, H, T, d, seed=1700 + d + m + W, dtype="bf16", scale="rms")
+    t["omega"] = synth.make_omega(d, m)
+    g = _cuda(t)
+    q, k, v, r, u, dO = (units(t[n]) for n in ("q", "k", "v", "r", "u", "dO"))
+    ref = C.bwd(q, k, v, r, u, to64(t["omega"]), W, dO)
+    # forward chain: remember what every segment started from
+    bounds, lo = [], 0
+    for hi in cuts:
+        bounds.append((lo, hi))
+        lo = hi
+    saved, state = [], None
+    for lo, hi in bounds:
+        seg = [g[n][:, :, lo:hi].contiguous() for n in ("q", "k", "v", "r", "u")]
+        nh = min(W - 1, lo)
+        hist = None if nh == 0 else (g["r"][:, :, lo - nh:lo].contiguous(), g["u"][:, :, lo - nh:lo].contiguous())
+        o, L, lse, S, z = P.fwd_continue(*seg, g["omega"], state=state, history=hist, W=W)
+        saved.append((seg, state, hist, L, lse))
+        state = (S, z)
+    # backward chain
+    grads = [torch.zeros(B, H, T, d, device="cuda", dtype=torch.float32) for _ in range(5)]
+    d_state = None
+    for (lo, hi), (seg, st, hist, L, lse) in reversed(list(zip(bounds, saved))):
+        dseg, dh, d_state = P.bwd_continue(*seg, g["omega"], L, lse, g["dO"][:, :, lo:hi].contiguous(), state=st,
+                                           history=hist, d_state=d_state, W=W)
+        for acc, part in zip(grads, dseg):
+            acc[:, :, lo:hi] += part.float()
+        if dh is not None:
+            nh = dh[0].shape[2]
+            grads[3][:, :, lo - nh:lo] += dh[0].float()
+            grads[4][:, :, lo - nh:lo] += dh[1].float()
+    torch.cuda.synchronize()
+    # the state before the first token is empty: nothing may depend on what flows into it, but it must be finite
+    assert torch.isfinite(d_state[0]).all() and torch.isfinite(d_state[1]).all()
+    for name, got, want in zip(("dq", "dk", "dv", "dr", "du"), grads, ref):
+        assert rel_err(units(got), want, floor=1e-2) <= 2e-2, name
+
+
+def test_state_gradient_of_a_continued_segment():
+    """dS_init, dz_init against the oracle: the gradient of sum(dO * o_segment) with respect to the state the segment
+    starts from, by central differences of the oracle's forward along random directions of (M0, a0)."""
+    B, H, T, d, m, W, T0 = 1, 2, 70, 64, 64, 64, 90
+    t = synth.make_inputs(B, H, T0 + T, d, seed=1811, dtype="bf16", scale="rms")
+    t["omega"] = synth.make_omega(d, m)
+    g = _cuda(t)
+    om = to64(t["omega"])
+    q, k, v, r, u, dO = (units(t[n]) for n in ("q", "k", "v", "r", "u", "dO"))
+    pre = [g[n][:, :, :T0].contiguous() for n in ("q", "k", "v", "r", "u")]
+    _, _, _, S0, z0 = P.fwd(*pre, g["omega"], W=W, return_state=True)
+    seg = [g[n][:, :, T0:].contiguous() for n in ("q", "k", "v", "r", "u")]
+    hist = (g["r"][:, :, T0 - (W - 1):T0].contiguous(), g["u"][:, :, T0 - (W - 1):T0].contiguous())
+    o, L, lse, S1, z1 = P.fwd_continue(*seg, g["omega"], state=(S0, z0), history=hist, W=W)
+    _, _, (dS0, dz0) = P.bwd_continue(*seg, g["omega"], L, lse, g["dO"][:, :, T0:].contiguous(), state=(S0, z0),
+                                      history=hist, W=W)
+    torch.cuda.synchronize()
+    # oracle: rows T0-(W-1) .. T0+T with the first W-1 as history, state (M0, a0) in its own convention (1/sqrt(m) inside)
+    M0 = to64(S0).reshape(B * H, m, d) / np.sqrt(m)
+    a0 = to64(z0).reshape(B * H, m) / np.sqrt(m)
+    sl = slice(T0 - (W - 1), T0 + T)
+    rng = np.random.default_rng(5)
+
+    def loss(Mx, ax):
+        oo = C.fwd(q[:, sl], k[:, sl], v[:, sl], r[:, sl], u[:, sl], om, W, 1e-30, M0=Mx, a0=ax, t0=W - 1)
+        return float((oo[:, W - 1:] * dO[:, T0:]).sum())
+
+    gS = to64(dS0).reshape(B * H, m, d) * np.sqrt(m)          # d/dM0 = sqrt(m) d/dS (S = sqrt(m) M)
+    gz = to64(dz0).reshape(B * H, m) * np.sqrt(m)
+    for _ in range(3):
+        # directions relative to each entry (the features' magnitudes span many orders): stays in the linear regime
+        dM = rng.standard_normal(M0.shape) * M0
+        da = rng.standard_normal(a0.shape) * a0
+        h = 1e-3
+        num = (loss(M0 + h * dM, a0 + h * da) - loss(M0 - h * dM, a0 - h * da)) / (2 * h)
+        ana = float((gS * dM).sum() + (gz * da).sum())
+        # a directional derivative is a sum of terms of both signs: the error is measured against their total size
+        scale = float(np.abs(gS * dM).sum() + np.abs(gz * da).sum())
+        assert abs(num - ana) <= 2e-2 * scale, (num, ana, scale)
+
+
 def test_prefill_then_decode_hand_off():
     # prefix by the forward, ring by linsimp_ring_fill, then single-token steps: the outputs must be the rows a
     # forward over the whole sequence gives
