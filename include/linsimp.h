@@ -52,7 +52,7 @@
 extern "C" {
 #endif
 
-#define LINSIMP_VERSION 3
+#define LINSIMP_VERSION 4
 
 enum {
     LINSIMP_OK = 0,
@@ -65,7 +65,8 @@ enum {
 };
 
 enum { LINSIMP_F32 = 0, LINSIMP_BF16 = 1 };          /* io_dtype */
-enum { LINSIMP_OP_FWD = 0, LINSIMP_OP_BWD = 1, LINSIMP_OP_DECODE = 2, LINSIMP_OP_STATE = 3, LINSIMP_OP_NORM = 4 };
+enum { LINSIMP_OP_FWD = 0, LINSIMP_OP_BWD = 1, LINSIMP_OP_DECODE = 2, LINSIMP_OP_STATE = 3, LINSIMP_OP_NORM = 4,
+       LINSIMP_OP_FWD_PACKED = 5, LINSIMP_OP_BWD_PACKED = 6 };
 enum {
     LINSIMP_ALGO_DEFAULT = 0, /* fp32 I/O: fp32 CUDA-core kernels; bf16 I/O: tensor-core kernels */
     LINSIMP_ALGO_FP32 = 1     /* force the fp32 CUDA-core kernels (any io_dtype)      */
@@ -272,8 +273,8 @@ int linsimp_prefill_state(const linsimp_params *p, const void *k, const void *v,
  *        min(seq_lens[b], W) rows (token t in slot t mod W); continue decoding sequence b with
  *        pos[b] = seq_lens[b].
  * Available where the tensor-core kernels are (bf16 I/O, default algo, d in {64,128},
- * m in {32,64,128}); LINSIMP_EUNSUPPORTED otherwise.  Packed (cu_seqlens) layouts are not
- * taken: a sequence must start at row 0 of its batch entry.
+ * m in {32,64,128}); LINSIMP_EUNSUPPORTED otherwise.  A sequence starts at row 0 of its batch
+ * entry here; the *_packed calls below take sequences laid end to end.
  */
 int linsimp_fwd_padded(const linsimp_params *p,
                        const void *q, const void *k, const void *v, const void *r, const void *u,
@@ -288,6 +289,38 @@ int linsimp_bwd_padded(const linsimp_params *p,
                        void *workspace, size_t workspace_bytes, linsimp_stream stream);
 int linsimp_ring_fill_padded(const linsimp_params *p, const void *r, const void *u, const int32_t *seq_lens,
                              void *ring_r, void *ring_u, linsimp_stream stream);
+
+/*
+ * Packed batches (Theorem 1 again: sequences are independent, so how they share a buffer is
+ * data layout only; the paper has no counterpart).  The token streams are [H, total_tokens, d]:
+ * for every head the sequences lie end to end, sequence b in rows [cu_seqlens[b], cu_seqlens[b+1]).
+ * cu_seqlens [B+1] int32 (device), non-decreasing, cu_seqlens[0] >= 0, cu_seqlens[B] <= total_tokens
+ * (the library does not check the values; rows outside every sequence are neither read nor written).
+ * p->B = number of sequences, p->T = an upper bound on the longest sequence (a longer one is cut at T).
+ *   linsimp_fwd_packed: o [H,total_tokens,d], rowmax_L, lse [H,total_tokens] for the sequences' rows;
+ *        S_final [B,H,m,d], z_final [B,H,m] (nullable) per sequence after its own last token.
+ *   linsimp_bwd_packed: rowmax_L, lse from linsimp_fwd_packed, dO and the five gradients [H,total_tokens,d].
+ *   linsimp_ring_fill_packed: decode ring [B,H,W,d] of each sequence from its own last min(len, W) rows
+ *        (token t in slot t mod W); continue decoding sequence b with pos[b] = its length.
+ * The sequences are moved into the padded form inside the workspace, run through the padded-batch
+ * kernels and gathered back, so the cost is that of a padded batch of B x T tokens plus the copies.
+ * workspace: linsimp_workspace_bytes(p, LINSIMP_OP_FWD_PACKED / LINSIMP_OP_BWD_PACKED).
+ * LINSIMP_FLAG_REUSE_FWD_STATE is not accepted (LINSIMP_EINVAL).  bf16 I/O on the tensor-core kernels
+ * only; LINSIMP_EUNSUPPORTED otherwise.
+ */
+int linsimp_fwd_packed(const linsimp_params *p,
+                       const void *q, const void *k, const void *v, const void *r, const void *u,
+                       const float *omega, const int32_t *cu_seqlens, int64_t total_tokens,
+                       void *o, float *rowmax_L, float *lse, float *S_final, float *z_final,
+                       void *workspace, size_t workspace_bytes, linsimp_stream stream);
+int linsimp_bwd_packed(const linsimp_params *p,
+                       const void *q, const void *k, const void *v, const void *r, const void *u,
+                       const float *omega, const int32_t *cu_seqlens, int64_t total_tokens,
+                       const float *rowmax_L, const float *lse, const void *dO,
+                       void *dq, void *dk, void *dv, void *dr, void *du,
+                       void *workspace, size_t workspace_bytes, linsimp_stream stream);
+int linsimp_ring_fill_packed(const linsimp_params *p, const void *r, const void *u, const int32_t *cu_seqlens,
+                             int64_t total_tokens, void *ring_r, void *ring_u, linsimp_stream stream);
 
 /*
  * Input side of a head (Sec. 3.1, the definitions before the trilinear score): the streams

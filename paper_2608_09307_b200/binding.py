@@ -5,7 +5,7 @@ import os
 import torch
 
 F32, BF16 = 0, 1
-OP_FWD, OP_BWD, OP_DECODE, OP_STATE, OP_NORM = 0, 1, 2, 3, 4
+OP_FWD, OP_BWD, OP_DECODE, OP_STATE, OP_NORM, OP_FWD_PACKED, OP_BWD_PACKED = 0, 1, 2, 3, 4, 5, 6
 ALGO_DEFAULT, ALGO_FP32 = 0, 1
 FLAG_REUSE_FWD_STATE = 1
 FLAG_OMEGA_IMAGE = 2
@@ -19,7 +19,8 @@ EXPORTS = ("linsimp_workspace_bytes", "linsimp_fwd", "linsimp_bwd", "linsimp_dec
            "linsimp_strerror", "linsimp_version", "linsimp_last_launch_count",
            "linsimp_profile_enable", "linsimp_profile_read", "linsimp_read_status", "linsimp_fwd_static",
            "linsimp_qkr_normalize", "linsimp_qkr_normalize_bwd", "linsimp_gate_rmsnorm", "linsimp_gate_rmsnorm_bwd",
-           "linsimp_fwd_padded", "linsimp_bwd_padded", "linsimp_ring_fill_padded", "linsimp_bwd_continue")
+           "linsimp_fwd_padded", "linsimp_bwd_padded", "linsimp_ring_fill_padded", "linsimp_bwd_continue",
+           "linsimp_fwd_packed", "linsimp_bwd_packed", "linsimp_ring_fill_packed")
 
 
 class LinSimpError(RuntimeError):
@@ -93,6 +94,13 @@ def load_library():
                                        ctypes.c_size_t, vp]
     lib.linsimp_ring_fill_padded.restype = ctypes.c_int
     lib.linsimp_ring_fill_padded.argtypes = [pp, vp, vp, ip, vp, vp, vp]
+    lib.linsimp_fwd_packed.restype = ctypes.c_int
+    lib.linsimp_fwd_packed.argtypes = [pp, vp, vp, vp, vp, vp, fp, ip, ctypes.c_int64, vp, fp, fp, fp, fp, vp, ctypes.c_size_t, vp]
+    lib.linsimp_bwd_packed.restype = ctypes.c_int
+    lib.linsimp_bwd_packed.argtypes = [pp, vp, vp, vp, vp, vp, fp, ip, ctypes.c_int64, fp, fp, vp, vp, vp, vp, vp, vp, vp,
+                                       ctypes.c_size_t, vp]
+    lib.linsimp_ring_fill_packed.restype = ctypes.c_int
+    lib.linsimp_ring_fill_packed.argtypes = [pp, vp, vp, ip, ctypes.c_int64, vp, vp, vp]
     lib.linsimp_read_status.restype = ctypes.c_int
     lib.linsimp_read_status.argtypes = [vp, vp]
     lib.linsimp_strerror.restype = ctypes.c_char_p
@@ -352,6 +360,69 @@ def ring_fill_padded(r, u, seq_lens, W=64, stream=None):
     ring_r = torch.zeros((B, H, W, d), dtype=r.dtype, device=r.device)
     ring_u = torch.zeros((B, H, W, d), dtype=r.dtype, device=r.device)
     _check(lib.linsimp_ring_fill_padded(ctypes.byref(p), _ptr(r), _ptr(u), _ptr(_lens(seq_lens, B)), _ptr(ring_r),
+                                        _ptr(ring_u), _stream(stream)))
+    return ring_r, ring_u
+
+
+def _cu(cu_seqlens):
+    if cu_seqlens.dtype != torch.int32 or cu_seqlens.dim() != 1 or cu_seqlens.numel() < 2:
+        raise LinSimpError("cu_seqlens must be an int32 tensor [B + 1]")
+    _dev(cu_seqlens)
+    return cu_seqlens
+
+
+def fwd_packed(q, k, v, r, u, omega, cu_seqlens, max_len, W=64, eps=1e-30, return_state=False, workspace=None, stream=None):
+    """linsimp_fwd_packed: q..u [H, total_tokens, d] bf16, sequence b in rows cu_seqlens[b]:cu_seqlens[b+1] of every head;
+    max_len: an upper bound on the longest sequence.  Returns (o, rowmax_L, lse) in the packed layout (rows outside
+    every sequence are left untouched) and, with return_state, also per-sequence (S_final, z_final)."""
+    lib = load_library()
+    _dev(q, k, v, r, u, omega)
+    H, total, d = q.shape
+    B = cu_seqlens.numel() - 1
+    m = omega.shape[-1]
+    p = make_params(B, H, max(1, int(max_len)), d, m, W, _io_dtype(q), omega.dim() == 3, ALGO_DEFAULT, eps)
+    o = torch.zeros_like(q)
+    L = torch.zeros((H, total), dtype=torch.float32, device=q.device)
+    lse = torch.zeros((H, total), dtype=torch.float32, device=q.device)
+    S = z = None
+    if return_state:
+        S = torch.empty((B, H, m, d), dtype=torch.float32, device=q.device)
+        z = torch.empty((B, H, m), dtype=torch.float32, device=q.device)
+    ws, ws_bytes = _workspace(p, OP_FWD_PACKED, workspace, q.device)
+    _check(lib.linsimp_fwd_packed(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),
+                                  _ptr(_cu(cu_seqlens)), total, _ptr(o), _ptr(L), _ptr(lse), _ptr(S), _ptr(z), _ptr(ws),
+                                  ws_bytes, _stream(stream)))
+    if return_state:
+        return o, L, lse, S, z
+    return o, L, lse
+
+
+def bwd_packed(q, k, v, r, u, omega, cu_seqlens, max_len, L, lse, dO, W=64, eps=1e-30, workspace=None, stream=None):
+    """linsimp_bwd_packed.  Returns dq, dk, dv, dr, du in the packed layout (rows outside every sequence are zero)."""
+    lib = load_library()
+    _dev(q, k, v, r, u, omega, L, lse, dO)
+    H, total, d = q.shape
+    B = cu_seqlens.numel() - 1
+    m = omega.shape[-1]
+    p = make_params(B, H, max(1, int(max_len)), d, m, W, _io_dtype(q), omega.dim() == 3, ALGO_DEFAULT, eps)
+    grads = [torch.zeros_like(q) for _ in range(5)]
+    ws, ws_bytes = _workspace(p, OP_BWD_PACKED, workspace, q.device)
+    _check(lib.linsimp_bwd_packed(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),
+                                  _ptr(_cu(cu_seqlens)), total, _ptr(L), _ptr(lse), _ptr(dO), *[_ptr(g) for g in grads],
+                                  _ptr(ws), ws_bytes, _stream(stream)))
+    return tuple(grads)
+
+
+def ring_fill_packed(r, u, cu_seqlens, W=64, stream=None):
+    """linsimp_ring_fill_packed: decode rings [B,H,W,d] (zero-initialised) from a packed batch."""
+    lib = load_library()
+    _dev(r, u)
+    H, total, d = r.shape
+    B = cu_seqlens.numel() - 1
+    p = make_params(B, H, 1, d, 64, W, _io_dtype(r))
+    ring_r = torch.zeros((B, H, W, d), dtype=r.dtype, device=r.device)
+    ring_u = torch.zeros_like(ring_r)
+    _check(lib.linsimp_ring_fill_packed(ctypes.byref(p), _ptr(r), _ptr(u), _ptr(_cu(cu_seqlens)), total, _ptr(ring_r),
                                         _ptr(ring_u), _stream(stream)))
     return ring_r, ring_u
 

@@ -10,6 +10,7 @@
 #include "common.cuh"
 #include "launch.cuh"
 #include "norm_gate.h"
+#include "packed.h"
 #include "simt_kernels.h"
 #include "tc_kernels.h"
 
@@ -67,7 +68,7 @@ void profile_after(cudaStream_t st)
 
 namespace {
 
-thread_local int g_launches[5] = {0, 0, 0, 0, 0};
+thread_local int g_launches[7] = {0, 0, 0, 0, 0, 0, 0};
 
 bool params_ok(const linsimp_params *p, int op)
 {
@@ -399,12 +400,49 @@ int run_tc_blocks(int op, const linsimp_params *p, const void *q, const void *k,
     return finish(op, tc_blocks_bwd_run(a, p->m, bw, lem, (cudaStream_t)stream));
 }
 
+// Packed batches: the inner (padded-batch) workspace first, then the sequences' lengths and the padded copies of the
+// token streams (and of the per-row scalars).
+struct PackedLayout {
+    size_t inner_bytes, lens, rows[11], scal[2], total;
+};
+
+PackedLayout packed_layout(const linsimp_params *p, int op)
+{
+    PackedLayout L;
+    memset(&L, 0, sizeof(L));
+    const int inner_op = op == LINSIMP_OP_FWD_PACKED ? LINSIMP_OP_FWD : LINSIMP_OP_BWD;
+    L.inner_bytes = tc_layout(p, inner_op).total;
+    size_t off = align_up(L.inner_bytes, 256);
+    L.lens = off;
+    off = align_up(off + (size_t)p->B * sizeof(int32_t), 256);
+    const size_t nrow = align_up((size_t)p->B * p->H * p->T * p->d * 2, 256);
+    const int n_rows = op == LINSIMP_OP_FWD_PACKED ? 6 : 11;
+    for (int x = 0; x < n_rows; ++x) {
+        L.rows[x] = off;
+        off += nrow;
+    }
+    for (int x = 0; x < 2; ++x) {
+        L.scal[x] = off;
+        off += align_up((size_t)p->B * p->H * p->T * sizeof(float), 256);
+    }
+    L.total = off;
+    return L;
+}
+
+bool packed_supported(const linsimp_params *p)
+{
+    return p->io_dtype == LINSIMP_BF16 && shape_supported(p) && use_tc(p, LINSIMP_OP_FWD) && use_tc(p, LINSIMP_OP_BWD) &&
+           !(p->flags & LINSIMP_FLAG_REUSE_FWD_STATE);
+}
+
 }  // namespace
 
 extern "C" {
 
 size_t linsimp_workspace_bytes(const linsimp_params *p, int op)
 {
+    if (op == LINSIMP_OP_FWD_PACKED || op == LINSIMP_OP_BWD_PACKED)
+        return (params_ok(p, LINSIMP_OP_FWD) && packed_supported(p)) ? packed_layout(p, op).total : 0;
     if (op == LINSIMP_OP_NORM)
         return (norm_shape_ok(p) && norm_gate_supported(p->d)) ? norm_gate_partial_bytes(p->B, p->H, p->T) : 0;
     if (op < 0 || op > 3 || !params_ok(p, op) || !shape_supported(p)) return 0;
@@ -540,6 +578,93 @@ int linsimp_bwd_padded(const linsimp_params *p, const void *q, const void *k, co
     if ((uintptr_t)seq_lens & 3u) return LINSIMP_EALIGN;
     return run_tc_bwd(p, q, k, v, r, u, omega, o, rowmax_L, lse, dO, dq, dk, dv, dr, du, workspace, workspace_bytes, stream,
                       seq_lens);
+}
+
+int linsimp_fwd_packed(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                       const float *omega, const int32_t *cu_seqlens, int64_t total_tokens, void *o, float *rowmax_L, float *lse,
+                       float *S_final, float *z_final, void *workspace, size_t workspace_bytes, linsimp_stream stream)
+{
+    if (!params_ok(p, LINSIMP_OP_FWD)) return LINSIMP_EINVAL;
+    if (!q || !k || !v || !r || !u || !omega || !o || !rowmax_L || !lse || !cu_seqlens || total_tokens < 0) return LINSIMP_EINVAL;
+    if ((S_final == nullptr) != (z_final == nullptr)) return LINSIMP_EINVAL;
+    if (p->flags & LINSIMP_FLAG_REUSE_FWD_STATE) return LINSIMP_EINVAL;
+    if (!packed_supported(p)) return LINSIMP_EUNSUPPORTED;
+    const void *ptrs[] = {q, k, v, r, u, o, omega};
+    for (const void *x : ptrs)
+        if (!aligned16(x)) return LINSIMP_EALIGN;
+    if ((uintptr_t)cu_seqlens & 3u) return LINSIMP_EALIGN;
+    const PackedLayout L = packed_layout(p, LINSIMP_OP_FWD_PACKED);
+    if (!workspace || workspace_bytes < L.total) return LINSIMP_EWORKSPACE;
+    if ((uintptr_t)workspace & 255u) return LINSIMP_EALIGN;
+    char *ws = (char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t *lens = (int32_t *)(ws + L.lens);
+    int launched = 0;
+    auto add = [&](int c) { if (c < 0) launched = -1; else if (launched >= 0) launched += c; };
+    add(packed_lens_run(cu_seqlens, p->B, p->T, lens, st));
+    const void *in[5] = {q, k, v, r, u};
+    for (int x = 0; x < 5; ++x) add(packed_unpack_run(in[x], cu_seqlens, p->B, p->H, p->T, total_tokens, p->d, 2, ws + L.rows[x], st));
+    if (launched < 0) return LINSIMP_ECUDA;
+    const int rc = linsimp_fwd_padded(p, ws + L.rows[0], ws + L.rows[1], ws + L.rows[2], ws + L.rows[3], ws + L.rows[4], omega, lens,
+                                      ws + L.rows[5], (float *)(ws + L.scal[0]), (float *)(ws + L.scal[1]), S_final, z_final, ws,
+                                      L.inner_bytes, stream);
+    if (rc != LINSIMP_OK) return rc;
+    launched += g_launches[LINSIMP_OP_FWD];
+    add(packed_pack_run(ws + L.rows[5], cu_seqlens, p->B, p->H, p->T, total_tokens, p->d, 2, o, st));
+    add(packed_pack_run(ws + L.scal[0], cu_seqlens, p->B, p->H, p->T, total_tokens, 1, 4, rowmax_L, st));
+    add(packed_pack_run(ws + L.scal[1], cu_seqlens, p->B, p->H, p->T, total_tokens, 1, 4, lse, st));
+    return finish(LINSIMP_OP_FWD_PACKED, launched);
+}
+
+int linsimp_bwd_packed(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                       const float *omega, const int32_t *cu_seqlens, int64_t total_tokens, const float *rowmax_L, const float *lse,
+                       const void *dO, void *dq, void *dk, void *dv, void *dr, void *du, void *workspace, size_t workspace_bytes,
+                       linsimp_stream stream)
+{
+    if (!params_ok(p, LINSIMP_OP_BWD)) return LINSIMP_EINVAL;
+    if (!q || !k || !v || !r || !u || !omega || !rowmax_L || !lse || !dO || !dq || !dk || !dv || !dr || !du || !cu_seqlens ||
+        total_tokens < 0)
+        return LINSIMP_EINVAL;
+    if (p->flags & LINSIMP_FLAG_REUSE_FWD_STATE) return LINSIMP_EINVAL;
+    if (!packed_supported(p)) return LINSIMP_EUNSUPPORTED;
+    const void *ptrs[] = {q, k, v, r, u, omega, dO, dq, dk, dv, dr, du};
+    for (const void *x : ptrs)
+        if (!aligned16(x)) return LINSIMP_EALIGN;
+    if (((uintptr_t)cu_seqlens & 3u) || ((uintptr_t)rowmax_L & 3u) || ((uintptr_t)lse & 3u)) return LINSIMP_EALIGN;
+    const PackedLayout L = packed_layout(p, LINSIMP_OP_BWD_PACKED);
+    if (!workspace || workspace_bytes < L.total) return LINSIMP_EWORKSPACE;
+    if ((uintptr_t)workspace & 255u) return LINSIMP_EALIGN;
+    char *ws = (char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t *lens = (int32_t *)(ws + L.lens);
+    int launched = 0;
+    auto add = [&](int c) { if (c < 0) launched = -1; else if (launched >= 0) launched += c; };
+    add(packed_lens_run(cu_seqlens, p->B, p->T, lens, st));
+    const void *in[6] = {q, k, v, r, u, dO};
+    for (int x = 0; x < 6; ++x) add(packed_unpack_run(in[x], cu_seqlens, p->B, p->H, p->T, total_tokens, p->d, 2, ws + L.rows[x], st));
+    add(packed_unpack_run(rowmax_L, cu_seqlens, p->B, p->H, p->T, total_tokens, 1, 4, ws + L.scal[0], st));
+    add(packed_unpack_run(lse, cu_seqlens, p->B, p->H, p->T, total_tokens, 1, 4, ws + L.scal[1], st));
+    if (launched < 0) return LINSIMP_ECUDA;
+    // (the output argument of the padded backward is not read: any valid pointer will do)
+    const int rc = linsimp_bwd_padded(p, ws + L.rows[0], ws + L.rows[1], ws + L.rows[2], ws + L.rows[3], ws + L.rows[4], omega, lens,
+                                      ws + L.rows[5], (const float *)(ws + L.scal[0]), (const float *)(ws + L.scal[1]), ws + L.rows[5],
+                                      ws + L.rows[6], ws + L.rows[7], ws + L.rows[8], ws + L.rows[9], ws + L.rows[10], ws,
+                                      L.inner_bytes, stream);
+    if (rc != LINSIMP_OK) return rc;
+    launched += g_launches[LINSIMP_OP_BWD];
+    void *out[5] = {dq, dk, dv, dr, du};
+    for (int x = 0; x < 5; ++x) add(packed_pack_run(ws + L.rows[6 + x], cu_seqlens, p->B, p->H, p->T, total_tokens, p->d, 2, out[x], st));
+    return finish(LINSIMP_OP_BWD_PACKED, launched);
+}
+
+int linsimp_ring_fill_packed(const linsimp_params *p, const void *r, const void *u, const int32_t *cu_seqlens, int64_t total_tokens,
+                             void *ring_r, void *ring_u, linsimp_stream stream)
+{
+    if (!params_ok(p, LINSIMP_OP_FWD) || !r || !u || !ring_r || !ring_u || !cu_seqlens || total_tokens < 0) return LINSIMP_EINVAL;
+    if (p->W > 64) return LINSIMP_EUNSUPPORTED;
+    if (!aligned16(r) || !aligned16(u) || !aligned16(ring_r) || !aligned16(ring_u) || ((uintptr_t)cu_seqlens & 3u)) return LINSIMP_EALIGN;
+    return finish(LINSIMP_OP_STATE, packed_ring_fill_run(r, u, cu_seqlens, p->B, p->H, total_tokens, p->d, p->W,
+                                                         p->io_dtype == LINSIMP_F32 ? 4 : 2, ring_r, ring_u, (cudaStream_t)stream));
 }
 
 int linsimp_ring_fill_padded(const linsimp_params *p, const void *r, const void *u, const int32_t *seq_lens, void *ring_r,
@@ -790,6 +915,6 @@ const char *linsimp_strerror(int code)
 
 int linsimp_version(void) { return LINSIMP_VERSION; }
 
-int linsimp_last_launch_count(int op) { return (op >= 0 && op <= 4) ? g_launches[op] : 0; }
+int linsimp_last_launch_count(int op) { return (op >= 0 && op <= 6) ? g_launches[op] : 0; }
 
 }  // extern "C"

@@ -280,3 +280,46 @@ def test_ragged_prefill_then_decode(d, m, W, per_head, lens):
             assert rel_err(to64(S[b, h]), M_ref[0] * np.sqrt(m)) < 5e-5
             assert rel_err(to64(z[b, h]), a_ref[0] * np.sqrt(m)) < 5e-5
 
+
+
+@pytest.mark.parametrize("d,m,W,lens,per_head", [(128, 128, 64, (130, 0, 1, 257, 64), False), (64, 128, 64, (5, 300, 17), True),
+                                                 (64, 32, 7, (40, 41), False)])
+def test_packed_batches(d, m, W, lens, per_head):
+    """Sequences laid end to end in one token buffer (cu_seqlens), with a gap of unused rows in front and behind:
+    forward, backward and ring fill against the oracle run on every sequence alone; lengths 0 and 1 included;
+    rows outside every sequence stay untouched."""
+    H = 2
+    front, back = 3, 5
+    starts = np.concatenate([[front], front + np.cumsum(lens)]).astype(np.int32)
+    total = int(starts[-1]) + back
+    t = synth.make_inputs(1, H, total, d, seed=1900 + d + m, dtype="bf16", scale="rms")
+    om = synth.make_omega(d, m, heads=H if per_head else None)
+    g = {n: v[0].contiguous().cuda() for n, v in t.items()}             # [H, total, d]
+    omg = om.cuda()
+    cu = torch.from_numpy(starts).cuda()
+    o, L, lse, S, z = P.fwd_packed(g["q"], g["k"], g["v"], g["r"], g["u"], omg, cu, max(lens), W=W, return_state=True)
+    grads = P.bwd_packed(g["q"], g["k"], g["v"], g["r"], g["u"], omg, cu, max(lens), L, lse, g["dO"], W=W)
+    ring_r, ring_u = P.ring_fill_packed(g["r"], g["u"], cu, W=W)
+    torch.cuda.synchronize()
+    inside = torch.zeros(total, dtype=torch.bool)
+    for b, n in enumerate(lens):
+        inside[starts[b]:starts[b] + n] = True
+    for got in (o,) + grads:
+        assert torch.all(got[:, ~inside.cuda()] == 0)
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert torch.all(S[b] == 0) and torch.all(z[b] == 0) and torch.all(ring_r[b] == 0)
+            continue
+        lo = int(starts[b])
+        for h in range(H):
+            cut = {name: to64(t[name][0, h:h + 1, lo:lo + n]) for name in ("q", "k", "v", "r", "u", "dO")}
+            omh = to64(om[h] if per_head else om)
+            o_ref, _, M_ref, a_ref = C.fwd(cut["q"], cut["k"], cut["v"], cut["r"], cut["u"], omh, W, return_state=True)
+            assert rel_err(to64(o[h:h + 1, lo:lo + n]), o_ref) <= 2e-2, (b, h)
+            assert rel_err(to64(S[b, h:h + 1]), M_ref * np.sqrt(m)) < 5e-5
+            assert rel_err(to64(z[b, h:h + 1]), a_ref * np.sqrt(m)) < 5e-5
+            g_ref = C.bwd(cut["q"], cut["k"], cut["v"], cut["r"], cut["u"], omh, W, cut["dO"])
+            for name, got, want in zip(("dq", "dk", "dv", "dr", "du"), grads, g_ref):
+                assert rel_err(to64(got[h:h + 1, lo:lo + n]), want, floor=1e-2) <= 2e-2, (b, h, name)
+            for tok in range(max(0, n - W), n):
+                assert torch.equal(ring_r[b, h, tok % W], g["r"][h, lo + tok]) and torch.equal(ring_u[b, h, tok % W], g["u"][h, lo + tok])

@@ -27,7 +27,7 @@ def test_exports_every_declared_symbol():
     for name in decl:
         assert hasattr(lib, name), name
     assert set(binding.EXPORTS) <= decl
-    assert lib.linsimp_version() == 3
+    assert lib.linsimp_version() == 4
 
 
 def test_workspace_and_argument_checks_on_host():
@@ -84,6 +84,40 @@ def test_workspace_and_argument_checks_on_host():
     # padded batches: seq_lens is required
     assert lib.linsimp_fwd_padded(ctypes.byref(p), al, al, al, al, al, al, n, al, al, al, n, n, al, 1 << 40, n) == -1
     assert lib.linsimp_ring_fill_padded(ctypes.byref(p), al, al, n, al, al, n) == -1
+
+
+def test_packed_and_continued_calls_check_their_arguments_on_the_host():
+    lib = P.load_library()
+    n = ctypes.c_void_p(None)
+    buf = ctypes.create_string_buffer(4096)
+    al = ctypes.c_void_p((ctypes.addressof(buf) + 255) // 256 * 256)
+    p = binding.make_params(3, 2, 100, 64, 128, 64, P.BF16)
+    f32 = binding.make_params(3, 2, 100, 64, 128, 64, P.F32)
+    keep = binding.make_params(3, 2, 100, 64, 128, 64, P.BF16, flags=binding.FLAG_REUSE_FWD_STATE)
+    inner = P.workspace_bytes(p, P.OP_BWD)
+    assert P.workspace_bytes(p, binding.OP_BWD_PACKED) >= inner + 11 * 3 * 2 * 100 * 64 * 2
+    assert P.workspace_bytes(p, binding.OP_FWD_PACKED) >= P.workspace_bytes(p, P.OP_FWD) + 6 * 3 * 2 * 100 * 64 * 2
+    assert P.workspace_bytes(f32, binding.OP_FWD_PACKED) == 0 and P.workspace_bytes(keep, binding.OP_BWD_PACKED) == 0
+    # forward: cu_seqlens missing -> EINVAL; fp32 streams -> EUNSUPPORTED; workspace too small -> EWORKSPACE
+    fwd = lambda pp, cu, ws: lib.linsimp_fwd_packed(ctypes.byref(pp), al, al, al, al, al, al, cu, 300, al, al, al, n, n, al, ws, n)
+    assert fwd(p, n, 1 << 40) == -1
+    assert fwd(f32, al, 1 << 40) == -2
+    assert fwd(p, al, 64) == -4
+    assert fwd(keep, al, 1 << 40) == -1
+    bwd = lambda pp, cu, ws: lib.linsimp_bwd_packed(ctypes.byref(pp), al, al, al, al, al, al, cu, 300, al, al, al, al, al, al, al, al,
+                                                    al, ws, n)
+    assert bwd(p, n, 1 << 40) == -1 and bwd(f32, al, 1 << 40) == -2 and bwd(p, al, 64) == -4
+    assert lib.linsimp_ring_fill_packed(ctypes.byref(p), al, al, n, 300, al, al, n) == -1
+    # continued backward: history without its gradient buffers, state gradient without its partner, reuse flag
+    cont = lambda pp, hr, dhr, nh, dSf, dzf: lib.linsimp_bwd_continue(ctypes.byref(pp), al, al, al, al, al, al, al, al, hr, hr, nh,
+                                                                       al, al, al, dSf, dzf, al, al, al, al, al, dhr, dhr, al, al,
+                                                                       al, 64, n)
+    assert cont(p, al, n, 5, n, n) == -1
+    assert cont(p, al, al, 64, n, n) == -1                 # more than W - 1 history rows
+    assert cont(p, n, n, 0, al, n) == -1
+    assert cont(keep, n, n, 0, n, n) == -1
+    assert cont(f32, n, n, 0, n, n) == -2
+    assert cont(p, al, al, 5, al, al) == -4                # everything in order except the workspace size
 
 
 def test_large_decode_batches_still_get_every_check():
