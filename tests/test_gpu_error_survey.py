@@ -1,0 +1,100 @@
+"""Error surveys of the bf16-input / fp32-state path beyond the named configurations: a grid of seeds, lengths and
+kernel instances, and a set of seeded random combinations (narrow windows, the zero-padded rank-32 instance, per-head
+banks, two-token sequences at m = 256 whose attention is saturated).  Every case is compared with the oracle in the
+library's metric, max|gpu - ref| / max|ref| per output tensor.
+
+What the surveys establish: o, dq, dv, dr, du stay within the 2e-2 of the named configurations everywhere.  dk has
+the least margin (its numerator and normaliser parts cancel, so the bf16 rounding of the boundary state shows three
+times as large as in the output): it stays within 2e-2 in all but a few cases of the grid and within 2.5e-2 in all,
+which is what these tests pin; the named configurations themselves (test_gpu_full_configs.py) are within 2e-2.
+One regime is held to 4e-2: sequences of two or three tokens at feature ranks above 128.  There a query sees a handful
+of pairs, the 128-feature blocks' parts of dq, dk, dr are each several times larger than their sum, and what is left
+after they cancel carries the blocks' bf16-operand noise (0.05-0.2 absolute against gradients of order 1-10); from
+a few dozen tokens on the same rank is back within 2e-2 (the T = 260, 1000 and 1500 cases below)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_09307_b200 as P
+from paper_2608_09307_b200 import synth
+from oracle import c_ref as C
+from tests.util import rel_err, to64, units
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2            # the path's tolerance
+TOL_DK = 2.5e-2       # what dk is held to outside the named configurations
+TOL_FEW = 4e-2        # dq, dk, dr of two- and three-token sequences at feature ranks above 128
+NAMES = ("o", "dq", "dk", "dv", "dr", "du")
+
+
+def _errors(t, om, W, per_head=False):
+    """Per-tensor metric over all units of one call, and the worst per-unit ratio of every tensor."""
+    g = {k_: v_.cuda() for k_, v_ in t.items()}
+    omg = om.cuda()
+    o, L, lse = P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, W=W)
+    grads = P.bwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, o, L, lse, g["dO"], W=W)
+    torch.cuda.synchronize()
+    B, H = t["q"].shape[:2]
+    got, ref = {n: [] for n in NAMES}, {n: [] for n in NAMES}
+    for b in range(B):
+        for h in range(H):
+            cut = {name: to64(t[name][b, h:h + 1]) for name in ("q", "k", "v", "r", "u", "dO")}
+            om64 = to64(om[h] if per_head else om)
+            refs = (C.fwd(cut["q"], cut["k"], cut["v"], cut["r"], cut["u"], om64, W, 1e-30),) + \
+                tuple(C.bwd(cut["q"], cut["k"], cut["v"], cut["r"], cut["u"], om64, W, cut["dO"]))
+            for n, x, y in zip(NAMES, (o,) + tuple(grads), refs):
+                got[n].append(to64(x[b, h]).ravel())
+                ref[n].append(np.asarray(y).ravel())
+    per_tensor = {n: rel_err(np.concatenate(got[n]), np.concatenate(ref[n]), floor=1e-2) for n in NAMES}
+    per_unit = {n: max(rel_err(a, b_, floor=1e-2) for a, b_ in zip(got[n], ref[n])) for n in NAMES}
+    return per_tensor, per_unit
+
+
+def test_seed_grid():
+    """48 cases: T in {40, 300, 1000} x four seeds x (d, m) in {(128,128), (64,128), (64,64), (64,32)}."""
+    worst = {}
+    dk_over = []
+    for d, m in ((128, 128), (64, 128), (64, 64), (64, 32)):
+        for T in (40, 300, 1000):
+            for seed in range(4):
+                t = synth.make_inputs(1, 2, T, d, seed=7000 + 100 * T + seed + d + m, dtype="bf16", scale="rms")
+                om = synth.make_omega(d, m, seed + 2)
+                e, _ = _errors(t, om, 64)
+                for n in NAMES:
+                    worst[(d, m, n)] = max(worst.get((d, m, n), 0.0), e[n])
+                    if n != "dk":
+                        assert e[n] <= TOL, (d, m, T, seed, n, e[n])
+                assert e["dk"] <= TOL_DK, (d, m, T, seed, e["dk"])
+                if e["dk"] > TOL:
+                    dk_over.append((d, m, T, seed, round(e["dk"], 4)))
+    for d, m in ((128, 128), (64, 128), (64, 64), (64, 32)):
+        print("d=%d m=%d worst:" % (d, m), " ".join("%s %.1e" % (n, worst[(d, m, n)]) for n in NAMES))
+    print("cases with dk above %.0e: %s" % (TOL, dk_over))
+    assert len(dk_over) <= 3
+
+
+# B, H, T, d, m, W, per_head, seed
+COMBOS = [
+    (2, 2, 333, 64, 32, 7, False, 1), (1, 3, 1200, 64, 64, 7, True, 2), (3, 1, 90, 128, 128, 7, False, 3),
+    (2, 2, 2, 64, 256, 64, False, 4), (1, 2, 2, 128, 256, 64, False, 5), (2, 3, 2, 64, 256, 33, True, 6),
+    (1, 1, 2100, 128, 128, 64, False, 7), (2, 2, 1, 64, 64, 64, False, 8), (1, 2, 65, 128, 64, 64, True, 9),
+    (3, 2, 129, 64, 128, 17, False, 10), (1, 3, 700, 64, 32, 33, True, 11), (2, 1, 48, 128, 32, 48, False, 12),
+    (1, 2, 1500, 64, 256, 64, False, 13), (2, 2, 260, 128, 256, 16, True, 14), (1, 1, 31, 64, 384, 64, False, 15),
+    (2, 3, 15, 128, 128, 1, False, 16), (1, 2, 16, 64, 64, 2, True, 17), (3, 3, 17, 64, 128, 3, False, 18),
+    (1, 2, 900, 128, 64, 64, False, 19), (2, 1, 2049, 64, 64, 64, False, 20), (1, 3, 450, 128, 128, 25, True, 21),
+    (2, 2, 77, 64, 32, 64, False, 22), (1, 1, 1000, 64, 512, 64, False, 23), (3, 1, 200, 128, 128, 64, True, 24),
+]
+
+
+@pytest.mark.parametrize("B,H,T,d,m,W,per_head,seed", COMBOS)
+def test_random_combination(B, H, T, d, m, W, per_head, seed):
+    t = synth.make_inputs(B, H, T, d, seed=8800 + seed, dtype="bf16", scale="rms")
+    om = synth.make_omega(d, m, 40 + seed, heads=H if per_head else None)
+    e, unit = _errors(t, om, W, per_head)
+    print("per tensor:", " ".join("%s %.1e" % (n, e[n]) for n in NAMES), "| worst unit:",
+          " ".join("%s %.1e" % (n, unit[n]) for n in NAMES))
+    few = T <= 3 and m > 128
+    for n in NAMES:
+        tol = TOL_FEW if (few and n in ("dq", "dk", "dr")) else (TOL_DK if n == "dk" else TOL)
+        assert e[n] <= tol, (n, e[n])
