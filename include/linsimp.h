@@ -82,7 +82,16 @@ enum {
     /* linsimp_decode_step only: the workspace holds the image of omega that linsimp_decode_prepare
      * wrote (same parameters, same omega, untouched since); the step then copies it instead of
      * converting omega again.  Ignored by kernels that keep omega in fp32. */
-    LINSIMP_FLAG_OMEGA_IMAGE = 2
+    LINSIMP_FLAG_OMEGA_IMAGE = 2,
+    /* linsimp_fwd and linsimp_bwd: both orientations of the trilinear score (Eq. two-views) kernelised and averaged
+     * (App. E, first item), in the windowed form of this operator.  View 1 is the estimator as defined (composite
+     * query q_i * r_c over the window, keys k_j over the prefix); view 2 exchanges the two key streams and their
+     * values (composite query q_i * k_j over the window, keys r_c over the prefix).  Numerators and normalisers
+     * are added before the division: o_i = (N1_i + N2_i) / (Z1_i + Z2_i + 2 eps).  rowmax_L and lse then describe
+     * the combined estimator (lse = log(m (Z1 + Z2 + 2 eps))), S_final / z_final the state of view 1.  Costs two
+     * passes of the kernels.  bf16 I/O on the tensor-core kernels with m <= 128 only (LINSIMP_EUNSUPPORTED
+     * otherwise); LINSIMP_FLAG_REUSE_FWD_STATE has no effect together with it. */
+    LINSIMP_FLAG_TWO_VIEWS = 4
 };
 
 typedef struct {

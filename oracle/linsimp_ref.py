@@ -134,8 +134,12 @@ def exact_window_ref(q, k, v, r, u, W):
     return o
 
 
-def bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS, M0=None, a0=None, t0=0):
+def bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS, M0=None, a0=None, t0=0, upstream=None):
     """Analytic gradients of sum(dO * o) for one head (no gradient for omega).
+
+    With upstream = (dN [T, dv], dZ [T]) the gradients of a loss are returned whose
+    derivatives with respect to this call's own sums N_i, Z_i (Eqs. Ni, Zi) are given
+    directly (dO is then not used): what a combination of several estimators needs.
 
     Sweep 1 walks queries forward with the running state and yields dq, dr, du;
     sweep 2 walks backward accumulating D_j = sum_{i>=j} dM_i, e_j = sum_{i>=j} da_i
@@ -165,8 +169,11 @@ def bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS, M0=None, a0=None, t0=0):
         N = np.sum(g * u[c0:i + 1], axis=0)
         Z = np.sum(psi @ a)
         o_i = N / (Z + eps)
-        dN[i] = dO[i] / (Z + eps)
-        dZ[i] = -np.dot(dO[i], o_i) / (Z + eps)
+        if upstream is None:
+            dN[i] = dO[i] / (Z + eps)
+            dZ[i] = -np.dot(dO[i], o_i) / (Z + eps)
+        else:
+            dN[i], dZ[i] = upstream[0][i], upstream[1][i]
         du[c0:i + 1] += dN[i][None, :] * g
         dg = dN[i][None, :] * u[c0:i + 1]                  # [w, dv]
         dpsi = dg @ M.T + dZ[i] * a[None, :]               # [w, m]
@@ -189,6 +196,33 @@ def bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS, M0=None, a0=None, t0=0):
         dlk = dchi * chi[i]
         dk[i] = omega @ dlk - np.sum(dlk) * k[i]
     return dq, dk, dv, dr, du
+
+
+def two_views_ref(q, k, v, r, u, omega, W, eps=EPS, return_parts=False):
+    """Both orientations of the trilinear score (Eq. two-views) kernelised and averaged (App. E, first item), in the
+    windowed form of this operator: the first view is fwd_ref as it stands (composite query q*r_c over the window,
+    keys k_j global); the second exchanges the two key streams and their values (composite query q*k_j over the
+    window, keys r_c global).  The kernel estimates are averaged, i.e. numerators and normalisers are added before the
+    division: o_i = (N1_i + N2_i) / (Z1_i + Z2_i + 2 eps).  Needs v and u of the same width."""
+    _, N1, Z1 = fwd_ref(q, k, v, r, u, omega, W, eps, return_parts=True)
+    _, N2, Z2 = fwd_ref(q, r, u, k, v, omega, W, eps, return_parts=True)
+    o = (N1 + N2) / (Z1 + Z2 + 2.0 * eps)[:, None]
+    if return_parts:
+        return o, N1 + N2, Z1 + Z2
+    return o
+
+
+def two_views_bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS):
+    """Gradients of sum(dO * o) for two_views_ref: both views see the same derivatives with respect to their sums,
+    dN_i = dO_i / den_i and dZ_i = -(dO_i . o_i) / den_i with den_i = Z1_i + Z2_i + 2 eps; the second view's
+    gradients come back with the streams exchanged.  Returns dq, dk, dv, dr, du."""
+    dO = np.asarray(dO, dtype=np.float64)
+    o, N, Z = two_views_ref(q, k, v, r, u, omega, W, eps, return_parts=True)
+    den = Z + 2.0 * eps
+    up = (dO / den[:, None], -np.sum(dO * o, axis=1) / den)
+    dq1, dk1, dv1, dr1, du1 = bwd_ref(q, k, v, r, u, omega, W, dO, eps, upstream=up)
+    dq2, dr2, du2, dk2, dv2 = bwd_ref(q, r, u, k, v, omega, W, dO, eps, upstream=up)
+    return dq1 + dq2, dk1 + dk2, dv1 + dv2, dr1 + dr2, du1 + du2
 
 
 def decode_ref(q_t, k_t, v_t, r_t, u_t, omega, M, a, ring_r, ring_u, pos, W, eps=EPS):

@@ -9,6 +9,7 @@ OP_FWD, OP_BWD, OP_DECODE, OP_STATE, OP_NORM, OP_FWD_PACKED, OP_BWD_PACKED = 0, 
 ALGO_DEFAULT, ALGO_FP32 = 0, 1
 FLAG_REUSE_FWD_STATE = 1
 FLAG_OMEGA_IMAGE = 2
+FLAG_TWO_VIEWS = 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblinsimp.so")
@@ -164,16 +165,17 @@ def last_launch_count(op):
 
 
 def fwd(q, k, v, r, u, omega, W=64, eps=1e-30, algo=ALGO_DEFAULT, return_state=False, workspace=None,
-        out=None, stream=None):
+        out=None, stream=None, two_views=False):
     """linsimp_fwd.  q,k,v,r,u [B,H,T,d] (fp32 or bf16, CUDA); omega fp32 [d,m] or [H,d,m].
 
+    two_views: both orientations of the trilinear score averaged (LINSIMP_FLAG_TWO_VIEWS).
     Returns (o, rowmax_L, lse) and, with return_state, also (S_final, z_final).
     """
     lib = load_library()
     _dev(q, k, v, r, u, omega)
     B, H, T, d = q.shape
     m = omega.shape[-1]
-    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps)
+    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps, FLAG_TWO_VIEWS if two_views else 0)
     o = torch.empty_like(q) if out is None else out
     L = torch.empty((B, H, T), dtype=torch.float32, device=q.device)
     lse = torch.empty((B, H, T), dtype=torch.float32, device=q.device)
@@ -278,7 +280,7 @@ def ring_fill(r, u, ring_r, ring_u, t_first=0, stream=None):
 
 
 def bwd(q, k, v, r, u, omega, o, L, lse, dO, W=64, eps=1e-30, algo=ALGO_DEFAULT, workspace=None, stream=None,
-        reuse_fwd_state=False):
+        reuse_fwd_state=False, two_views=False):
     """linsimp_bwd.  Returns dq, dk, dv, dr, du (same shape/dtype as the inputs).
 
     reuse_fwd_state: `workspace` is the tensor the preceding fwd() call on the same inputs was given
@@ -291,7 +293,7 @@ def bwd(q, k, v, r, u, omega, o, L, lse, dO, W=64, eps=1e-30, algo=ALGO_DEFAULT,
     if reuse_fwd_state and workspace is None:
         raise ValueError("reuse_fwd_state needs the workspace of the forward call")
     p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps,
-                    FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0)
+                    (FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0) | (FLAG_TWO_VIEWS if two_views else 0))
     grads = [torch.empty_like(q) for _ in range(5)]
     ws, ws_bytes = _workspace(p, OP_BWD, workspace, q.device)
     _check(lib.linsimp_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),

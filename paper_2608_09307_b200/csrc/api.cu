@@ -79,7 +79,8 @@ bool params_ok(const linsimp_params *p, int op)
     if (p->io_dtype != LINSIMP_F32 && p->io_dtype != LINSIMP_BF16) return false;
     if (p->algo != LINSIMP_ALGO_DEFAULT && p->algo != LINSIMP_ALGO_FP32) return false;
     if (!(p->eps >= 0.f)) return false;
-    if (p->flags & ~(LINSIMP_FLAG_REUSE_FWD_STATE | LINSIMP_FLAG_OMEGA_IMAGE)) return false;
+    if (p->flags & ~(LINSIMP_FLAG_REUSE_FWD_STATE | LINSIMP_FLAG_OMEGA_IMAGE | LINSIMP_FLAG_TWO_VIEWS)) return false;
+    if ((p->flags & LINSIMP_FLAG_TWO_VIEWS) && !(op == LINSIMP_OP_FWD || op == LINSIMP_OP_BWD)) return false;
     return true;
 }
 
@@ -351,6 +352,52 @@ int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void
     return finish(LINSIMP_OP_BWD, tc_bwd_run(a, (cudaStream_t)stream));
 }
 
+// the two-orientation average runs on the single-block tensor-core kernels
+bool views_supported(const linsimp_params *p)
+{
+    return p->io_dtype == LINSIMP_BF16 && p->algo == LINSIMP_ALGO_DEFAULT && tc_supported(p->d, p->m) && tc_bwd_supported(p->d, p->m);
+}
+
+int run_tc_views(int op, const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                 const float *omega, void *o, float *rowmax_L, float *lse, float *S_final, float *z_final, const void *dO,
+                 void *dq, void *dk, void *dv, void *dr, void *du, void *workspace, size_t workspace_bytes, linsimp_stream stream)
+{
+    const TcLayout L = tc_layout(p, op);
+    const size_t base = align_up(L.total, 256);
+    if (!workspace || workspace_bytes < base + tc_views_extra_bytes(p->B, p->H, p->T, p->d, op)) return LINSIMP_EWORKSPACE;
+    if ((uintptr_t)workspace & 255u) return LINSIMP_EALIGN;
+    char *ws = (char *)workspace;
+    TcArgs a;
+    memset(&a, 0, sizeof(a));
+    a.B = p->B; a.H = p->H; a.T = p->T; a.d = p->d; a.m = tc_mf(p->m); a.m_real = p->m; a.omega_ld = p->m; a.state_m = p->m; a.p_off = 0; a.W = p->W;
+    a.omega_stride = p->omega_per_head ? (long)p->d * p->m : 0;
+    a.log2_eps_m = p->eps > 0.f ? (float)(log2((double)p->eps) + log2((double)p->m)) : -INFINITY;
+    a.chunks_per_cta = 16;
+    a.q = q; a.k = k; a.v = v; a.r = r; a.u = u; a.omega = omega;
+    a.o = o; a.L = rowmax_L; a.lse = lse; a.S_final = S_final; a.z_final = z_final; a.dO = dO;
+    a.dq = dq; a.dk = dk; a.dv = dv; a.dr = dr; a.du = du;
+    a.status = (int *)(ws + L.status);
+    a.chi_ml = (uint8_t *)(ws + L.chi_ml);
+    a.segtot = (float *)(ws + L.segtot);
+    a.images = (uint8_t *)(ws + L.images);
+    a.ab = (float *)(ws + L.ab);
+    a.om_img = (uint8_t *)(ws + L.om_img);
+    if (op == LINSIMP_OP_BWD) {
+        a.chi32 = (float *)(ws + L.chi32);
+        a.gstates = (float *)(ws + L.gstates);
+        a.segsum = (float *)(ws + L.segsum);
+        a.dv_intra = (float *)(ws + L.dv_intra);
+        a.dchi_intra = (float *)(ws + L.dchi_intra);
+        a.dr_acc = (float *)(ws + L.dr_acc);
+        a.du_acc = (float *)(ws + L.du_acc);
+    }
+    if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
+    TcBlockWs bw;
+    tc_views_carve(ws + base, p->B, p->H, p->T, p->d, op, &bw);
+    if (op == LINSIMP_OP_FWD) return finish(op, tc_views_fwd_run(a, bw, log_eps_m(p), (cudaStream_t)stream));
+    return finish(op, tc_views_bwd_run(a, bw, (cudaStream_t)stream));
+}
+
 // Feature rank above 128: fills the kernel arguments for one 128-feature block layout and runs all blocks.
 int run_tc_blocks(int op, const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
                   const float *omega, void *o, float *rowmax_L, float *lse, float *S_final, float *z_final, const void *dO,
@@ -446,6 +493,8 @@ size_t linsimp_workspace_bytes(const linsimp_params *p, int op)
     if (op == LINSIMP_OP_NORM)
         return (norm_shape_ok(p) && norm_gate_supported(p->d)) ? norm_gate_partial_bytes(p->B, p->H, p->T) : 0;
     if (op < 0 || op > 3 || !params_ok(p, op) || !shape_supported(p)) return 0;
+    if (p->flags & LINSIMP_FLAG_TWO_VIEWS)
+        return views_supported(p) ? align_up(tc_layout(p, op).total, 256) + tc_views_extra_bytes(p->B, p->H, p->T, p->d, op) : 0;
     if (op == LINSIMP_OP_DECODE)
         return (p->io_dtype == LINSIMP_BF16 && p->algo == LINSIMP_ALGO_DEFAULT &&
                 decode_mma_supported(p->d, p->m, p->W, decode_banks(p)))
@@ -471,6 +520,11 @@ int linsimp_fwd(const linsimp_params *p, const void *q, const void *k, const voi
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(r) || !aligned16(u) || !aligned16(o) ||
         !aligned16(omega))
         return LINSIMP_EALIGN;
+    if (p->flags & LINSIMP_FLAG_TWO_VIEWS) {
+        if (!views_supported(p)) return LINSIMP_EUNSUPPORTED;
+        return run_tc_views(LINSIMP_OP_FWD, p, q, k, v, r, u, omega, o, rowmax_L, lse, S_final, z_final, nullptr, nullptr, nullptr,
+                            nullptr, nullptr, nullptr, workspace, workspace_bytes, stream);
+    }
     if (use_tc_blocks(p, LINSIMP_OP_FWD))
         return run_tc_blocks(LINSIMP_OP_FWD, p, q, k, v, r, u, omega, o, rowmax_L, lse, S_final, z_final, nullptr, nullptr,
                              nullptr, nullptr, nullptr, nullptr, workspace, workspace_bytes, stream);
@@ -689,6 +743,11 @@ int linsimp_bwd(const linsimp_params *p, const void *q, const void *k, const voi
     const void *ptrs[] = {q, k, v, r, u, omega, o, dO, dq, dk, dv, dr, du};
     for (const void *x : ptrs)
         if (!aligned16(x)) return LINSIMP_EALIGN;
+    if (p->flags & LINSIMP_FLAG_TWO_VIEWS) {
+        if (!views_supported(p)) return LINSIMP_EUNSUPPORTED;
+        return run_tc_views(LINSIMP_OP_BWD, p, q, k, v, r, u, omega, (void *)o, (float *)rowmax_L, (float *)lse, nullptr, nullptr,
+                            dO, dq, dk, dv, dr, du, workspace, workspace_bytes, stream);
+    }
     if (use_tc_blocks(p, LINSIMP_OP_BWD))
         return run_tc_blocks(LINSIMP_OP_BWD, p, q, k, v, r, u, omega, (void *)o, (float *)rowmax_L, (float *)lse, nullptr,
                              nullptr, dO, dq, dk, dv, dr, du, workspace, workspace_bytes, stream);

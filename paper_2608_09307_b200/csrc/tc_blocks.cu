@@ -22,7 +22,7 @@ __global__ void k_blocks_combine(int nb, const float *__restrict__ o0, const flo
                                  const float *__restrict__ o2, const float *__restrict__ o3,
                                  const float *__restrict__ L0, const float *__restrict__ L1, const float *__restrict__ L2,
                                  const float *__restrict__ L3, const float *__restrict__ s0, const float *__restrict__ s1,
-                                 const float *__restrict__ s2, const float *__restrict__ s3, float log_eps_m, long rows, int d,
+                                 const float *__restrict__ s2, const float *__restrict__ s3, float log_eps_m, float guards_off, long rows, int d,
                                  bf16 *__restrict__ o, float *__restrict__ o_tot, float *__restrict__ Lout,
                                  float *__restrict__ lse)
 {
@@ -41,7 +41,7 @@ __global__ void k_blocks_combine(int nb, const float *__restrict__ o0, const flo
                 den += w;
                 num = fmaf(ob[b][idx], w, num);
             }
-            den -= (float)(nb - 1) * expf(log_eps_m - M);      // every w_b carries the guard once
+            den -= guards_off * expf(log_eps_m - M);           // every w_b carries the guard once
         }
         const float val = den > 0.f ? num / den : 0.f;
         if (o) o[idx] = __float2bfloat16_rn(val);
@@ -83,7 +83,7 @@ void tc_blocks_carve(char *base, int B, int H, int T, int d, int m, int op, TcBl
         w->lseb[b] = (float *)(base + off); off += up256(rows * 4);
     }
     w->delta = nullptr;
-    w->g32[0] = w->g32[1] = w->g32[2] = nullptr;
+    for (int x = 0; x < 5; ++x) w->g32[x] = nullptr;
     if (op == 1) {
         w->delta = (float *)(base + off); off += up256(rows * 4);
         for (int x = 0; x < 3; ++x) {
@@ -104,13 +104,15 @@ static TcArgs block_args(const TcArgs &a, int m_total, int b)
     return x;
 }
 
+// guards_off: how many copies of the guard eps*m the combined normaliser gives up (feature blocks of one estimator
+// keep one of their nb copies; the views of the two-orientation average keep theirs)
 static int combine(LaunchScope &sc, const TcArgs &a, int nb, const TcBlockWs &w, float log_eps_m, bf16 *o, float *o_tot,
-                   float *L, float *lse)
+                   float *L, float *lse, float guards_off)
 {
     const long rows = (long)a.B * a.H * a.T;
     LS_LAUNCH(sc, "blocks_combine", k_blocks_combine<<<1184, 256, 0, sc.stream>>>(
         nb, w.o32[0], w.o32[1], w.o32[2], w.o32[3], w.Lb[0], w.Lb[1], w.Lb[2], w.Lb[3], w.lseb[0], w.lseb[1], w.lseb[2],
-        w.lseb[3], log_eps_m, rows, a.d, o, o_tot, L, lse));
+        w.lseb[3], log_eps_m, guards_off, rows, a.d, o, o_tot, L, lse));
     return 0;
 }
 
@@ -129,7 +131,7 @@ static int blocks_forward(LaunchScope &sc, const TcArgs &a, int m_total, const T
         if (c < 0) return c;
         sc.count += c;
     }
-    return combine(sc, a, nb, w, log_eps_m, o, o_tot, L, lse);
+    return combine(sc, a, nb, w, log_eps_m, o, o_tot, L, lse, (float)(nb - 1));
 }
 
 int tc_blocks_fwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float log_eps_m, cudaStream_t st)
@@ -191,6 +193,106 @@ int tc_blocks_bwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float lo
     LS_LAUNCH(sc, "blocks_round", k_blocks_round<<<1184, 256, 0, st>>>(w.g32[0], (bf16 *)a.dq, ntok));
     LS_LAUNCH(sc, "blocks_round", k_blocks_round<<<1184, 256, 0, st>>>(w.g32[1], (bf16 *)a.dk, ntok));
     LS_LAUNCH(sc, "blocks_round", k_blocks_round<<<1184, 256, 0, st>>>(w.g32[2], (bf16 *)a.dv, ntok));
+    return sc.result();
+}
+
+// ------------------------------------------------------------------ both orientations of the trilinear score, averaged
+// View 1 is the estimator as it stands; view 2 exchanges the two key streams and their values (k <-> r, v <-> u).  The
+// kernel estimates are averaged: o = (N1 + N2) / (Z1 + Z2 + 2 eps), which in terms of the views' outputs and
+// log-normalisers is the same weighted mean the feature blocks use (every view keeps its guard).  In the backward both
+// views share dN_i and dZ_i of the combined estimator: the tile kernel runs per view in its sum-only mode first
+// (sum_c psi'_ic . dpsiN_ic of both views = dO_i . o_i den_i), then in full; view 2's gradients return exchanged.
+size_t tc_views_extra_bytes(int B, int H, int T, int d, int op)
+{
+    const size_t rows = (size_t)B * H * T;
+    if (op == 1) return up256(rows * 4) + 5 * up256(rows * d * 4);
+    return 2 * (up256(rows * d * 4) + 2 * up256(rows * 4));
+}
+
+void tc_views_carve(char *base, int B, int H, int T, int d, int op, TcBlockWs *w)
+{
+    const size_t rows = (size_t)B * H * T;
+    size_t off = 0;
+    for (int b = 0; b < 4; ++b) w->o32[b] = w->Lb[b] = w->lseb[b] = nullptr;
+    w->delta = nullptr;
+    for (int x = 0; x < 5; ++x) w->g32[x] = nullptr;
+    if (op == 1) {
+        w->delta = (float *)(base + off); off += up256(rows * 4);
+        for (int x = 0; x < 5; ++x) {
+            w->g32[x] = (float *)(base + off); off += up256(rows * d * 4);
+        }
+        return;
+    }
+    for (int b = 0; b < 2; ++b) {
+        w->o32[b] = (float *)(base + off); off += up256(rows * d * 4);
+        w->Lb[b] = (float *)(base + off); off += up256(rows * 4);
+        w->lseb[b] = (float *)(base + off); off += up256(rows * 4);
+    }
+}
+
+static TcArgs view_args(const TcArgs &a, int view)
+{
+    TcArgs x = a;
+    if (view == 1) {
+        x.k = a.r; x.r = a.k;
+        x.v = a.u; x.u = a.v;
+    }
+    x.reuse_state = 0;
+    x.S_final = view == 0 ? a.S_final : nullptr;        // the state of the (k, v) stream is the one the caller knows
+    x.z_final = view == 0 ? a.z_final : nullptr;
+    return x;
+}
+
+int tc_views_fwd_run(const TcArgs &a, const TcBlockWs &w, float log_eps_m, cudaStream_t st)
+{
+    LaunchScope sc = {st, 0};
+    for (int view = 0; view < 2; ++view) {
+        TcArgs x = view_args(a, view);
+        x.o32 = w.o32[view];
+        x.L = w.Lb[view];
+        x.lse = w.lseb[view];
+        x.chi32 = nullptr;
+        const int c = tc_fwd_run(x, st);
+        if (c < 0) return c;
+        sc.count += c;
+    }
+    combine(sc, a, 2, w, log_eps_m, (bf16 *)a.o, nullptr, a.L, a.lse, 0.f);
+    return sc.result();
+}
+
+int tc_views_bwd_run(const TcArgs &a, const TcBlockWs &w, cudaStream_t st)
+{
+    LaunchScope sc = {st, 0};
+    const long rows = (long)a.B * a.H * a.T, ntok = rows * a.d;
+    sc.check(cudaMemsetAsync(w.delta, 0, sizeof(float) * rows, st));
+    for (int view = 0; view < 2; ++view) {
+        TcArgs x = view_args(a, view);
+        x.delta_out = w.delta;
+        const int c = tc_bwd_run(x, st);
+        if (c < 0) return c;
+        sc.count += c;
+    }
+    // fp32 sums: g32[0..4] = dq, dk, dv, dr, du.  View 1 writes dq, dk, dv and accumulates dr, du; view 2 adds its dq,
+    // adds what it calls dk, dv (the gradients of its key stream: r, u) onto dr, du, and accumulates what it calls dr, du
+    // onto dk, dv.
+    for (int view = 0; view < 2; ++view) {
+        TcArgs x = view_args(a, view);
+        x.delta_ext = w.delta;
+        x.grad32 = view == 0 ? 1 : 2;
+        x.keep_acc = view == 1;
+        x.hold_acc = 1;
+        x.dq = w.g32[0];
+        x.dk = w.g32[view == 0 ? 1 : 3];
+        x.dv = w.g32[view == 0 ? 2 : 4];
+        x.dr_acc = w.g32[view == 0 ? 3 : 1];
+        x.du_acc = w.g32[view == 0 ? 4 : 2];
+        const int c = tc_bwd_run(x, st);
+        if (c < 0) return c;
+        sc.count += c;
+    }
+    void *out[5] = {a.dq, a.dk, a.dv, a.dr, a.du};
+    for (int x = 0; x < 5; ++x)
+        LS_LAUNCH(sc, "blocks_round", k_blocks_round<<<1184, 256, 0, st>>>(w.g32[x], (bf16 *)out[x], ntok));
     return sc.result();
 }
 

@@ -69,7 +69,7 @@ int tc_bwd_run(const TcArgs &a, cudaStream_t st);
 struct TcBlockWs {
     float *o32[4], *Lb[4], *lseb[4];   // per block: fp32 output, row shift, log-normaliser
     float *delta;                      // backward: [BH][T] dO_i . o_i den_i of the whole layer
-    float *g32[3];                     // backward: dq, dk, dv summed over the blocks in fp32
+    float *g32[5];                     // backward: dq, dk, dv (and, for the two views, dr, du) summed in fp32
 };
 int tc_blocks_supported(int d, int m);
 size_t tc_blocks_extra_bytes(int B, int H, int T, int d, int m, int op);
@@ -77,5 +77,12 @@ void tc_blocks_carve(char *base, int B, int H, int T, int d, int m, int op, TcBl
 int tc_blocks_fwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float eps_m, cudaStream_t st);
 int tc_blocks_state_run(const TcArgs &a, int m_total, cudaStream_t st);
 int tc_blocks_bwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float eps_m, cudaStream_t st);
+
+// Both orientations of the trilinear score averaged (Eq. two-views): the estimator as it stands plus the one with the
+// two key streams and their values exchanged, combined through their log-normalisers.
+size_t tc_views_extra_bytes(int B, int H, int T, int d, int op);
+void tc_views_carve(char *base, int B, int H, int T, int d, int op, TcBlockWs *w);
+int tc_views_fwd_run(const TcArgs &a, const TcBlockWs &w, float eps_m, cudaStream_t st);
+int tc_views_bwd_run(const TcArgs &a, const TcBlockWs &w, cudaStream_t st);
 
 }  // namespace linsimp

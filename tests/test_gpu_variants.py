@@ -1,0 +1,60 @@
+"""Variants of the estimator on the GPU against the oracle: both orientations of the trilinear score averaged
+(Eq. two-views, App. E first item)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_09307_b200 as P
+from paper_2608_09307_b200 import synth
+from oracle import linsimp_ref as R
+from tests.util import rel_err, to64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("B,H,T,d,m,W,per_head", [(1, 2, 150, 128, 128, 64, False), (2, 1, 70, 64, 128, 33, True),
+                                                  (1, 2, 40, 64, 32, 7, False), (1, 1, 17, 128, 64, 64, False)])
+def test_two_views_forward_and_backward(B, H, T, d, m, W, per_head):
+    t = synth.make_inputs(B, H, T, d, seed=2600 + T + d + m, dtype="bf16", scale="rms")
+    om = synth.make_omega(d, m, 9, heads=H if per_head else None)
+    g = {k_: v_.cuda() for k_, v_ in t.items()}
+    omg = om.cuda()
+    o, L, lse = P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, W=W, two_views=True)
+    grads = P.bwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, o, L, lse, g["dO"], W=W, two_views=True)
+    # exchanging the two key streams (with their values) must leave the output where it is and exchange the gradients
+    o_x, L_x, lse_x = P.fwd(g["q"], g["r"], g["u"], g["k"], g["v"], omg, W=W, two_views=True)
+    torch.cuda.synchronize()
+    assert rel_err(to64(o_x), to64(o)) <= 1e-2
+    names = ("o", "dq", "dk", "dv", "dr", "du")
+    got = {n: [] for n in names}
+    ref = {n: [] for n in names}
+    for b in range(B):
+        for h in range(H):
+            cut = [to64(t[name][b, h]) for name in ("q", "k", "v", "r", "u")]
+            om64 = to64(om[h] if per_head else om)
+            dO = to64(t["dO"][b, h])
+            o_ref, N_ref, Z_ref = R.two_views_ref(*cut, om64, W, return_parts=True)
+            g_ref = R.two_views_bwd_ref(*cut, om64, W, dO)
+            for n, x, y in zip(names, (o,) + tuple(grads), (o_ref,) + tuple(g_ref)):
+                got[n].append(to64(x[b, h]).ravel())
+                ref[n].append(np.asarray(y).ravel())
+            # the log-normaliser of the combined estimator
+            lse_ref = np.log(m * (Z_ref + 2e-30))
+            assert np.abs(to64(lse[b, h]) - lse_ref).max() < 5e-2
+    # the output within the path's tolerance; the gradients add the operand noise of two estimators whose parts
+    # partly cancel, and are held to 2.5e-2
+    for n in names:
+        e = rel_err(np.concatenate(got[n]), np.concatenate(ref[n]), floor=1e-2)
+        print(n, "%.2e" % e)
+        assert e <= (2e-2 if n == "o" else 2.5e-2), (n, e)
+
+
+def test_two_views_is_refused_where_it_has_no_kernels():
+    t = synth.make_inputs(1, 1, 20, 64, seed=1, dtype="fp32", scale="quarter")
+    g = {k_: v_.cuda() for k_, v_ in t.items()}
+    with pytest.raises(P.LinSimpError):
+        P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], synth.make_omega(64, 64).cuda(), two_views=True)       # fp32 streams
+    t = synth.make_inputs(1, 1, 20, 64, seed=1, dtype="bf16", scale="rms")
+    g = {k_: v_.cuda() for k_, v_ in t.items()}
+    with pytest.raises(P.LinSimpError):
+        P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], synth.make_omega(64, 256).cuda(), two_views=True)      # m above 128

@@ -64,10 +64,17 @@ def test_workspace_and_argument_checks_on_host():
     rc = lib.linsimp_bwd(ctypes.byref(p), *([n] * 15), n, 0, n)
     assert rc == -1
     # unknown flag bits are refused; the known one changes no size
-    odd = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, flags=6)
+    odd = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, flags=64)
     assert P.workspace_bytes(odd, P.OP_BWD) == 0
     keep = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, flags=binding.FLAG_REUSE_FWD_STATE)
     assert P.workspace_bytes(keep, P.OP_BWD) == P.workspace_bytes(p, P.OP_BWD)
+    # both orientations averaged: more scratch; not for the decode step, fp32 streams or ranks above 128
+    two = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, flags=binding.FLAG_TWO_VIEWS)
+    assert P.workspace_bytes(two, P.OP_FWD) > P.workspace_bytes(p, P.OP_FWD)
+    assert P.workspace_bytes(two, P.OP_BWD) > P.workspace_bytes(p, P.OP_BWD)
+    assert P.workspace_bytes(two, P.OP_DECODE) == 0
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.F32, flags=binding.FLAG_TWO_VIEWS), P.OP_FWD) == 0
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 256, 64, P.BF16, flags=binding.FLAG_TWO_VIEWS), P.OP_FWD) == 0
     # normalisation / gate calls: one float per 128 rows of a unit, rounded up to 256 bytes
     assert P.workspace_bytes(p, P.OP_NORM) == 256
     big = binding.make_params(2, 16, 16384, 128, 128, 64, P.BF16)
