@@ -52,7 +52,7 @@
 extern "C" {
 #endif
 
-#define LINSIMP_VERSION 4
+#define LINSIMP_VERSION 5
 
 enum {
     LINSIMP_OK = 0,
@@ -105,6 +105,11 @@ typedef struct {
     int32_t algo;             /* LINSIMP_ALGO_*                                       */
     float   eps;              /* guard of Eq. linearized-output, 1e-30 in the paper   */
     int32_t flags;            /* LINSIMP_FLAG_* bits, 0 for none                      */
+    int32_t dv;               /* width D_v of v, u (and o, dO, dv, du, S) when it differs from d (Sec. 3.1: q,k,r in
+                               * R^D, v,u in R^{D_v}); 0 or d: the same width.  Any D_v >= 1 with D_v * element size a
+                               * multiple of 16 bytes; taken by linsimp_fwd and linsimp_bwd only, where the layer runs
+                               * as ceil(D_v / d) blocks of d value channels (every value channel is an estimator of
+                               * its own that shares Z_i), at that many times the cost.  Other calls: LINSIMP_EINVAL. */
 } linsimp_params;
 
 typedef void *linsimp_stream;

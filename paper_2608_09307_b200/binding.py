@@ -33,7 +33,7 @@ class Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("T", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("m", ctypes.c_int32), ("W", ctypes.c_int32), ("io_dtype", ctypes.c_int32),
                 ("omega_per_head", ctypes.c_int32), ("algo", ctypes.c_int32), ("eps", ctypes.c_float),
-                ("flags", ctypes.c_int32)]
+                ("flags", ctypes.c_int32), ("dv", ctypes.c_int32)]
 
 
 def lib_path():
@@ -145,8 +145,8 @@ def _stream(stream):
     return ctypes.c_void_p(s.cuda_stream)
 
 
-def make_params(B, H, T, d, m, W, io_dtype, omega_per_head=False, algo=ALGO_DEFAULT, eps=1e-30, flags=0):
-    return Params(B, H, T, d, m, W, io_dtype, 1 if omega_per_head else 0, algo, eps, flags)
+def make_params(B, H, T, d, m, W, io_dtype, omega_per_head=False, algo=ALGO_DEFAULT, eps=1e-30, flags=0, dv=0):
+    return Params(B, H, T, d, m, W, io_dtype, 1 if omega_per_head else 0, algo, eps, flags, dv)
 
 
 def workspace_bytes(params, op):
@@ -175,13 +175,15 @@ def fwd(q, k, v, r, u, omega, W=64, eps=1e-30, algo=ALGO_DEFAULT, return_state=F
     _dev(q, k, v, r, u, omega)
     B, H, T, d = q.shape
     m = omega.shape[-1]
-    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps, FLAG_TWO_VIEWS if two_views else 0)
-    o = torch.empty_like(q) if out is None else out
+    dv = v.shape[-1]
+    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps, FLAG_TWO_VIEWS if two_views else 0,
+                    0 if dv == d else dv)
+    o = torch.empty_like(v) if out is None else out
     L = torch.empty((B, H, T), dtype=torch.float32, device=q.device)
     lse = torch.empty((B, H, T), dtype=torch.float32, device=q.device)
     S = z = None
     if return_state:
-        S = torch.empty((B, H, m, d), dtype=torch.float32, device=q.device)
+        S = torch.empty((B, H, m, dv), dtype=torch.float32, device=q.device)
         z = torch.empty((B, H, m), dtype=torch.float32, device=q.device)
     ws, ws_bytes = _workspace(p, OP_FWD, workspace, q.device)
     _check(lib.linsimp_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),
@@ -292,9 +294,11 @@ def bwd(q, k, v, r, u, omega, o, L, lse, dO, W=64, eps=1e-30, algo=ALGO_DEFAULT,
     m = omega.shape[-1]
     if reuse_fwd_state and workspace is None:
         raise ValueError("reuse_fwd_state needs the workspace of the forward call")
+    dv = v.shape[-1]
     p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps,
-                    (FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0) | (FLAG_TWO_VIEWS if two_views else 0))
-    grads = [torch.empty_like(q) for _ in range(5)]
+                    (FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0) | (FLAG_TWO_VIEWS if two_views else 0),
+                    0 if dv == d else dv)
+    grads = [torch.empty_like(x) for x in (q, k, v, r, u)]
     ws, ws_bytes = _workspace(p, OP_BWD, workspace, q.device)
     _check(lib.linsimp_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),
                            _ptr(o), _ptr(L), _ptr(lse), _ptr(dO), *[_ptr(g) for g in grads],

@@ -70,9 +70,16 @@ namespace {
 
 thread_local int g_launches[7] = {0, 0, 0, 0, 0, 0, 0};
 
-bool params_ok(const linsimp_params *p, int op)
+bool params_ok(const linsimp_params *p, int op, bool dv_taken = false)
 {
     if (!p) return false;
+    if (p->dv < 0) return false;
+    if (p->dv != 0 && p->dv != p->d) {
+        // a value width of its own: forward and backward only, rows of whole 16-byte pieces, no variant on top of it
+        if (!dv_taken) return false;
+        if (((size_t)p->dv * (p->io_dtype == LINSIMP_F32 ? 4 : 2)) % 16) return false;
+        if (p->flags & LINSIMP_FLAG_TWO_VIEWS) return false;
+    }
     if (p->B < 1 || p->H < 1 || p->d < 1 || p->m < 1 || p->W < 1) return false;
     if (op != LINSIMP_OP_DECODE && p->T < 1) return false;
     if (op != LINSIMP_OP_DECODE && (long long)p->B * p->H > 65535) return false;   // grid.y limit of the chunked kernels
@@ -482,12 +489,26 @@ bool packed_supported(const linsimp_params *p)
            !(p->flags & LINSIMP_FLAG_REUSE_FWD_STATE);
 }
 
+bool own_value_width(const linsimp_params *p) { return p->dv != 0 && p->dv != p->d; }
+
 }  // namespace
+
+namespace linsimp {
+size_t value_width_workspace_bytes(const linsimp_params *p, int op);
+int value_width_fwd(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                    const float *omega, void *o, float *rowmax_L, float *lse, float *S_final, float *z_final, void *workspace,
+                    size_t workspace_bytes, linsimp_stream stream, int *launched);
+int value_width_bwd(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
+                    const float *omega, const void *o, const float *rowmax_L, const float *lse, const void *dO, void *dq, void *dk,
+                    void *dv, void *dr, void *du, void *workspace, size_t workspace_bytes, linsimp_stream stream, int *launched);
+}  // namespace linsimp
 
 extern "C" {
 
 size_t linsimp_workspace_bytes(const linsimp_params *p, int op)
 {
+    if (p && own_value_width(p))
+        return ((op == LINSIMP_OP_FWD || op == LINSIMP_OP_BWD) && params_ok(p, op, true)) ? value_width_workspace_bytes(p, op) : 0;
     if (op == LINSIMP_OP_FWD_PACKED || op == LINSIMP_OP_BWD_PACKED)
         return (params_ok(p, LINSIMP_OP_FWD) && packed_supported(p)) ? packed_layout(p, op).total : 0;
     if (op == LINSIMP_OP_NORM)
@@ -513,13 +534,19 @@ int linsimp_fwd(const linsimp_params *p, const void *q, const void *k, const voi
                 const float *omega, void *o, float *rowmax_L, float *lse, float *S_final, float *z_final,
                 void *workspace, size_t workspace_bytes, linsimp_stream stream)
 {
-    if (!params_ok(p, LINSIMP_OP_FWD)) return LINSIMP_EINVAL;
+    if (!params_ok(p, LINSIMP_OP_FWD, true)) return LINSIMP_EINVAL;
     if (!q || !k || !v || !r || !u || !omega || !o || !rowmax_L || !lse) return LINSIMP_EINVAL;
     if ((S_final == nullptr) != (z_final == nullptr)) return LINSIMP_EINVAL;
     if (!shape_supported(p)) return LINSIMP_EUNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(r) || !aligned16(u) || !aligned16(o) ||
         !aligned16(omega))
         return LINSIMP_EALIGN;
+    if (own_value_width(p)) {
+        int extra = 0;
+        const int rc = value_width_fwd(p, q, k, v, r, u, omega, o, rowmax_L, lse, S_final, z_final, workspace, workspace_bytes, stream, &extra);
+        if (rc == LINSIMP_OK) g_launches[LINSIMP_OP_FWD] = g_launches[LINSIMP_OP_FWD] * ((p->dv + p->d - 1) / p->d) + extra;
+        return rc;
+    }
     if (p->flags & LINSIMP_FLAG_TWO_VIEWS) {
         if (!views_supported(p)) return LINSIMP_EUNSUPPORTED;
         return run_tc_views(LINSIMP_OP_FWD, p, q, k, v, r, u, omega, o, rowmax_L, lse, S_final, z_final, nullptr, nullptr, nullptr,
@@ -736,13 +763,20 @@ int linsimp_bwd(const linsimp_params *p, const void *q, const void *k, const voi
                 void *dq, void *dk, void *dv, void *dr, void *du, void *workspace, size_t workspace_bytes,
                 linsimp_stream stream)
 {
-    if (!params_ok(p, LINSIMP_OP_BWD)) return LINSIMP_EINVAL;
+    if (!params_ok(p, LINSIMP_OP_BWD, true)) return LINSIMP_EINVAL;
     if (!q || !k || !v || !r || !u || !omega || !o || !rowmax_L || !lse || !dO || !dq || !dk || !dv || !dr || !du)
         return LINSIMP_EINVAL;
     if (!shape_supported(p)) return LINSIMP_EUNSUPPORTED;
     const void *ptrs[] = {q, k, v, r, u, omega, o, dO, dq, dk, dv, dr, du};
     for (const void *x : ptrs)
         if (!aligned16(x)) return LINSIMP_EALIGN;
+    if (own_value_width(p)) {
+        int extra = 0;
+        const int rc = value_width_bwd(p, q, k, v, r, u, omega, o, rowmax_L, lse, dO, dq, dk, dv, dr, du, workspace, workspace_bytes,
+                                       stream, &extra);
+        if (rc == LINSIMP_OK) g_launches[LINSIMP_OP_BWD] = g_launches[LINSIMP_OP_BWD] * ((p->dv + p->d - 1) / p->d) + extra;
+        return rc;
+    }
     if (p->flags & LINSIMP_FLAG_TWO_VIEWS) {
         if (!views_supported(p)) return LINSIMP_EUNSUPPORTED;
         return run_tc_views(LINSIMP_OP_BWD, p, q, k, v, r, u, omega, (void *)o, (float *)rowmax_L, (float *)lse, nullptr, nullptr,

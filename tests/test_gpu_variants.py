@@ -58,3 +58,41 @@ def test_two_views_is_refused_where_it_has_no_kernels():
     g = {k_: v_.cuda() for k_, v_ in t.items()}
     with pytest.raises(P.LinSimpError):
         P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], synth.make_omega(64, 256).cuda(), two_views=True)      # m above 128
+
+
+@pytest.mark.parametrize("dtype,B,H,T,d,dv,m,W", [("bf16", 1, 2, 130, 64, 128, 128, 64), ("bf16", 2, 1, 90, 128, 64, 128, 64),
+                                                  ("bf16", 1, 1, 40, 64, 200, 64, 33), ("fp32", 1, 2, 50, 32, 48, 64, 7),
+                                                  ("bf16", 1, 2, 33, 128, 8, 128, 16)])
+def test_value_width_other_than_key_width(dtype, B, H, T, d, dv, m, W):
+    """v, u in R^{D_v}, q, k, r in R^D (Sec. 3.1): forward with final state and backward against the oracle."""
+    scale = "rms" if dtype == "bf16" else "quarter"
+    tk = synth.make_inputs(B, H, T, d, seed=2700 + d + dv, dtype=dtype, scale=scale, with_dO=False)
+    tv = synth.make_inputs(B, H, T, dv, seed=2800 + d + dv, dtype=dtype, scale=scale)
+    t = {"q": tk["q"], "k": tk["k"], "r": tk["r"], "v": tv["v"], "u": tv["u"], "dO": tv["dO"]}
+    om = synth.make_omega(d, m, 11)
+    g = {k_: v_.cuda() for k_, v_ in t.items()}
+    omg = om.cuda()
+    o, L, lse, S, z = P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, W=W, return_state=True)
+    grads = P.bwd(g["q"], g["k"], g["v"], g["r"], g["u"], omg, o, L, lse, g["dO"], W=W)
+    torch.cuda.synchronize()
+    assert o.shape == (B, H, T, dv) and S.shape == (B, H, m, dv)
+    assert grads[2].shape == (B, H, T, dv) and grads[4].shape == (B, H, T, dv) and grads[0].shape == (B, H, T, d)
+    tol = 2e-2 if dtype == "bf16" else 1e-4
+    names = ("o", "dq", "dk", "dv", "dr", "du")
+    got = {n: [] for n in names}
+    ref = {n: [] for n in names}
+    om64 = to64(om)
+    for b in range(B):
+        for h in range(H):
+            cut = [to64(t[name][b, h]) for name in ("q", "k", "v", "r", "u")]
+            o_ref = R.fwd_ref(*cut, om64, W)
+            g_ref = R.bwd_ref(*cut, om64, W, to64(t["dO"][b, h]))
+            for n, x, y in zip(names, (o,) + tuple(grads), (o_ref,) + tuple(g_ref)):
+                got[n].append(to64(x[b, h]).ravel())
+                ref[n].append(np.asarray(y).ravel())
+            M_ref, a_ref = R.prefix_state(cut[1], cut[2], om64)
+            assert rel_err(to64(S[b, h]), M_ref * np.sqrt(m)) < 5e-5
+            assert rel_err(to64(z[b, h]), a_ref * np.sqrt(m)) < 5e-5
+    for n in names:
+        e = rel_err(np.concatenate(got[n]), np.concatenate(ref[n]), floor=1e-2)
+        assert e <= (2.5e-2 if (n == "dk" and dtype == "bf16") else tol), (n, e)

@@ -27,7 +27,7 @@ def test_exports_every_declared_symbol():
     for name in decl:
         assert hasattr(lib, name), name
     assert set(binding.EXPORTS) <= decl
-    assert lib.linsimp_version() == 4
+    assert lib.linsimp_version() == 5
 
 
 def test_workspace_and_argument_checks_on_host():
@@ -125,6 +125,27 @@ def test_packed_and_continued_calls_check_their_arguments_on_the_host():
     assert cont(keep, n, n, 0, n, n) == -1
     assert cont(f32, n, n, 0, n, n) == -2
     assert cont(p, al, al, 5, al, al) == -4                # everything in order except the workspace size
+
+
+def test_value_width_is_taken_by_forward_and_backward_only():
+    lib = P.load_library()
+    n = ctypes.c_void_p(None)
+    buf = ctypes.create_string_buffer(4096)
+    al = ctypes.c_void_p((ctypes.addressof(buf) + 255) // 256 * 256)
+    same = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16)
+    wide = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, dv=160)       # three blocks of 64 value channels
+    assert P.workspace_bytes(wide, P.OP_FWD) > P.workspace_bytes(same, P.OP_FWD)
+    assert P.workspace_bytes(wide, P.OP_BWD) > P.workspace_bytes(same, P.OP_BWD)
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, dv=64), P.OP_FWD) == P.workspace_bytes(same, P.OP_FWD)
+    for op in (P.OP_DECODE, P.OP_STATE, binding.OP_FWD_PACKED):
+        assert P.workspace_bytes(wide, op) == 0
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, dv=100), P.OP_FWD) == 0     # rows of 200 bytes
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, dv=-8), P.OP_FWD) == 0
+    assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, dv=160, flags=binding.FLAG_TWO_VIEWS), P.OP_FWD) == 0
+    # calls that know one width only refuse the parameter
+    assert lib.linsimp_fwd_padded(ctypes.byref(wide), al, al, al, al, al, al, al, al, al, al, n, n, al, 1 << 40, n) == -1
+    assert lib.linsimp_decode_step(ctypes.byref(wide), *([al] * 13), 1 << 20, n) == -1
+    assert lib.linsimp_fwd(ctypes.byref(wide), al, al, al, al, al, al, al, al, al, n, n, al, 64, n) == -4
 
 
 def test_large_decode_batches_still_get_every_check():
