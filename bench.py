@@ -324,7 +324,36 @@ def bench_secondary(P, synth, torch, dev, steps, peaks):
     tf2 = fwd_flops_per_token_head(cfg2["d"], cfg2["m"], 64) * th2 / (ms2 * 1e-3) / 1e12
     c2 = dict(ms=ms2, tokens_per_s=cfg2["B"] * cfg2["T"] / (ms2 * 1e-3), tflops=tf2, **frac(tf2))
     del g2, ws2, o2
+    # the exact windowed 2-simplicial layer the paper compares with (joint softmax over 512 keys x 32 anchors), on the
+    # shapes of the main workload, forward only; unit-norm k and r and a query of norm 8 (a temperature), as that layer
+    # is run in the paper
+    gen = torch.Generator(device=dev).manual_seed(77)
+    Bw, Hw, Tw, dw = WORKLOAD["B"], WORKLOAD["H"], WORKLOAD["T"], WORKLOAD["d"]
+
+    def unit(scale):
+        x = torch.randn(Bw, Hw, Tw, dw, device=dev, generator=gen)
+        return (x / x.norm(dim=-1, keepdim=True) * scale).to(torch.bfloat16)
+
+    qw, kw, rw = unit(8.0), unit(1.0), unit(1.0)
+    vw, uw = unit(dw ** 0.5), unit(dw ** 0.5)
+    ow = torch.empty_like(qw)
+    for _ in range(3):
+        P.winsimp_fwd(qw, kw, vw, rw, uw, w1=512, w2=32, out=ow)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        P.winsimp_fwd(qw, kw, vw, rw, uw, w1=512, w2=32, out=ow)
+    e1.record()
+    torch.cuda.synchronize()
+    msw = e0.elapsed_time(e1) / steps
+    flw = 2.0 * 2.0 * 512 * 32 * dw * Bw * Hw * Tw          # score and value contraction over the full pair plane
+    tfw = flw / (msw * 1e-3) / 1e12
+    win = dict(ms=msw, tokens_per_s=Bw * Tw / (msw * 1e-3), tflops=tfw, finite=bool(torch.isfinite(ow.float()).all()), **frac(tfw))
+    del qw, kw, rw, vw, uw, ow
     return dict(steps=steps,
+                exact_windowed="exact 512 x 32 windowed 2-simplicial layer on B=%d H=%d T=%d d=%d bf16, fwd only "
+                               "(warp-level MMAs)" % (Bw, Hw, Tw, dw), winsimp=win,
                 c4_sweep="C4: B=4 H=8 T=8192 d=64 W=64 bf16, fwd+bwd, TFLOP/s in the 3x convention", c4=rows,
                 c2_forward="C2: B=8 H=16 T=4096 d=64 m=128 bf16, fwd only", c2=c2)
 

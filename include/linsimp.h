@@ -305,6 +305,21 @@ int linsimp_ring_fill_padded(const linsimp_params *p, const void *r, const void 
                              void *ring_r, void *ring_u, linsimp_stream stream);
 
 /*
+ * Exact windowed 2-simplicial attention, forward (the comparison layer of Sec. 4.3 "Baselines" and Table layouts: one
+ * joint softmax over a w1 x w2 pair plane, 512 x 32 in the paper's runs; Eq. exact-window-app with a window on the first
+ * key stream as well).  No random features, no state:
+ *     s_ijc = sum_a q_i[a] k_j[a] r_c[a],    o_i = sum_{j,c} exp(s_ijc) (v_j * u_c) / sum_{j,c} exp(s_ijc)
+ * over j in [max(0, i-w1+1), i] and c in [max(0, i-w2+1), i].  Inputs are used as given (normalisation and temperature
+ * are the caller's, as for linsimp_fwd).
+ *   in : q,k,v,r,u [B,H,T,d] bf16; p->W = w2 (1..32); w1 >= 1; p->d in {64,128}; p->m, p->eps unused
+ *   out: o [B,H,T,d] bf16; lse [B,H,T] fp32 (nullable): log of the normaliser
+ * No workspace.  fp32 streams, other widths or w2 > 32: LINSIMP_EUNSUPPORTED.
+ */
+int linsimp_winsimp_fwd(const linsimp_params *p, int32_t w1,
+                        const void *q, const void *k, const void *v, const void *r, const void *u,
+                        void *o, float *lse, linsimp_stream stream);
+
+/*
  * Packed batches (Theorem 1 again: sequences are independent, so how they share a buffer is
  * data layout only; the paper has no counterpart).  The token streams are [H, total_tokens, d]:
  * for every head the sequences lie end to end, sequence b in rows [cu_seqlens[b], cu_seqlens[b+1]).

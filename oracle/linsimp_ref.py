@@ -134,6 +134,26 @@ def exact_window_ref(q, k, v, r, u, W):
     return o
 
 
+def exact_two_window_ref(q, k, v, r, u, w1, w2, return_lse=False):
+    """Exact joint softmax over the pair plane j in [i-w1+1, i] x c in [i-w2+1, i] (the windowed exact layer the paper
+    compares with, Sec. 4.3 "Baselines": Eq. exact-window-app with a window on the key stream too), with the
+    trilinear score of Eq. trilinear-score on the inputs as given."""
+    q, k, v, r, u = (np.asarray(t, dtype=np.float64) for t in (q, k, v, r, u))
+    T, dv = q.shape[0], v.shape[1]
+    o = np.zeros((T, dv))
+    lse = np.zeros(T)
+    for i in range(T):
+        j0, c0 = max(0, i - w1 + 1), max(0, i - w2 + 1)
+        s = ((q[i][None, :] * r[c0:i + 1]) @ k[j0:i + 1].T)          # [anchors, keys]
+        mx = s.max()
+        kappa = np.exp(s - mx)
+        Z = kappa.sum()
+        G = kappa @ v[j0:i + 1]                                       # [anchors, dv]
+        o[i] = np.sum(G * u[c0:i + 1], axis=0) / Z
+        lse[i] = mx + np.log(Z)
+    return (o, lse) if return_lse else o
+
+
 def bwd_ref(q, k, v, r, u, omega, W, dO, eps=EPS, M0=None, a0=None, t0=0, upstream=None):
     """Analytic gradients of sum(dO * o) for one head (no gradient for omega).
 

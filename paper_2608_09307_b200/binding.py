@@ -21,7 +21,7 @@ EXPORTS = ("linsimp_workspace_bytes", "linsimp_fwd", "linsimp_bwd", "linsimp_dec
            "linsimp_profile_enable", "linsimp_profile_read", "linsimp_read_status", "linsimp_fwd_static",
            "linsimp_qkr_normalize", "linsimp_qkr_normalize_bwd", "linsimp_gate_rmsnorm", "linsimp_gate_rmsnorm_bwd",
            "linsimp_fwd_padded", "linsimp_bwd_padded", "linsimp_ring_fill_padded", "linsimp_bwd_continue",
-           "linsimp_fwd_packed", "linsimp_bwd_packed", "linsimp_ring_fill_packed")
+           "linsimp_fwd_packed", "linsimp_bwd_packed", "linsimp_ring_fill_packed", "linsimp_winsimp_fwd")
 
 
 class LinSimpError(RuntimeError):
@@ -102,6 +102,8 @@ def load_library():
                                        ctypes.c_size_t, vp]
     lib.linsimp_ring_fill_packed.restype = ctypes.c_int
     lib.linsimp_ring_fill_packed.argtypes = [pp, vp, vp, ip, ctypes.c_int64, vp, vp, vp]
+    lib.linsimp_winsimp_fwd.restype = ctypes.c_int
+    lib.linsimp_winsimp_fwd.argtypes = [pp, ctypes.c_int32, vp, vp, vp, vp, vp, vp, fp, vp]
     lib.linsimp_read_status.restype = ctypes.c_int
     lib.linsimp_read_status.argtypes = [vp, vp]
     lib.linsimp_strerror.restype = ctypes.c_char_p
@@ -368,6 +370,19 @@ def ring_fill_padded(r, u, seq_lens, W=64, stream=None):
     _check(lib.linsimp_ring_fill_padded(ctypes.byref(p), _ptr(r), _ptr(u), _ptr(_lens(seq_lens, B)), _ptr(ring_r),
                                         _ptr(ring_u), _stream(stream)))
     return ring_r, ring_u
+
+
+def winsimp_fwd(q, k, v, r, u, w1=512, w2=32, return_lse=False, out=None, stream=None):
+    """linsimp_winsimp_fwd: exact windowed 2-simplicial attention (joint softmax over w1 keys x w2 anchors), bf16."""
+    lib = load_library()
+    _dev(q, k, v, r, u)
+    B, H, T, d = q.shape
+    p = make_params(B, H, T, d, 64, w2, _io_dtype(q))
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, H, T), dtype=torch.float32, device=q.device) if return_lse else None
+    _check(lib.linsimp_winsimp_fwd(ctypes.byref(p), int(w1), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(o), _ptr(lse),
+                                   _stream(stream)))
+    return (o, lse) if return_lse else o
 
 
 def _cu(cu_seqlens):

@@ -494,6 +494,8 @@ bool own_value_width(const linsimp_params *p) { return p->dv != 0 && p->dv != p-
 }  // namespace
 
 namespace linsimp {
+int winsimp_run(const linsimp_params *p, int w1, const void *q, const void *k, const void *v, const void *r, const void *u, void *o,
+                float *lse, cudaStream_t st);
 size_t value_width_workspace_bytes(const linsimp_params *p, int op);
 int value_width_fwd(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,
                     const float *omega, void *o, float *rowmax_L, float *lse, float *S_final, float *z_final, void *workspace,
@@ -659,6 +661,20 @@ int linsimp_bwd_padded(const linsimp_params *p, const void *q, const void *k, co
     if ((uintptr_t)seq_lens & 3u) return LINSIMP_EALIGN;
     return run_tc_bwd(p, q, k, v, r, u, omega, o, rowmax_L, lse, dO, dq, dk, dv, dr, du, workspace, workspace_bytes, stream,
                       seq_lens);
+}
+
+int linsimp_winsimp_fwd(const linsimp_params *p, int32_t w1, const void *q, const void *k, const void *v, const void *r,
+                        const void *u, void *o, float *lse, linsimp_stream stream)
+{
+    if (!p || p->B < 1 || p->H < 1 || p->T < 1 || p->W < 1 || w1 < 1 || (long long)p->B * p->H > 65535) return LINSIMP_EINVAL;
+    if (!q || !k || !v || !r || !u || !o) return LINSIMP_EINVAL;
+    if ((p->dv != 0 && p->dv != p->d) || p->flags) return LINSIMP_EINVAL;
+    if (p->io_dtype != LINSIMP_BF16 || !(p->d == 64 || p->d == 128) || p->W > 32) return LINSIMP_EUNSUPPORTED;
+    const void *ptrs[] = {q, k, v, r, u, o};
+    for (const void *x : ptrs)
+        if (!aligned16(x)) return LINSIMP_EALIGN;
+    if ((uintptr_t)lse & 3u) return LINSIMP_EALIGN;
+    return finish(LINSIMP_OP_FWD, winsimp_run(p, w1, q, k, v, r, u, o, lse, (cudaStream_t)stream));
 }
 
 int linsimp_fwd_packed(const linsimp_params *p, const void *q, const void *k, const void *v, const void *r, const void *u,

@@ -96,3 +96,24 @@ def test_value_width_other_than_key_width(dtype, B, H, T, d, dv, m, W):
     for n in names:
         e = rel_err(np.concatenate(got[n]), np.concatenate(ref[n]), floor=1e-2)
         assert e <= (2.5e-2 if (n == "dk" and dtype == "bf16") else tol), (n, e)
+
+
+@pytest.mark.parametrize("B,H,T,d,w1,w2", [(1, 2, 700, 128, 512, 32), (2, 1, 300, 64, 512, 32), (1, 1, 130, 128, 64, 7),
+                                           (1, 2, 67, 64, 100, 1), (1, 1, 5, 128, 512, 32)])
+def test_exact_windowed_layer(B, H, T, d, w1, w2):
+    """linsimp_winsimp_fwd against the oracle's joint pair softmax (key window w1, anchor window w2), ragged tile tails,
+    windows longer than the sequence and a one-anchor window included."""
+    t = synth.make_inputs(B, H, T, d, seed=2900 + T + d, dtype="bf16", scale="rms", with_dO=False)
+    # the paper's regime for this layer: unit-norm k, r and a query scaled by a temperature (here 0.5 sqrt(d))
+    g = {}
+    for n_, sc in (("q", 0.5), ("k", d ** -0.5), ("r", d ** -0.5), ("v", 1.0), ("u", 1.0)):
+        t[n_] = (t[n_].float() * sc).to(torch.bfloat16)
+        g[n_] = t[n_].cuda()
+    o, lse = P.winsimp_fwd(g["q"], g["k"], g["v"], g["r"], g["u"], w1=w1, w2=w2, return_lse=True)
+    torch.cuda.synchronize()
+    for b in range(B):
+        for h in range(H):
+            cut = [to64(t[name][b, h]) for name in ("q", "k", "v", "r", "u")]
+            o_ref, lse_ref = R.exact_two_window_ref(*cut, w1, w2, return_lse=True)
+            assert rel_err(to64(o[b, h]), o_ref) <= 2e-2, (b, h)
+            assert np.abs(to64(lse[b, h]) - lse_ref).max() < 5e-2
