@@ -331,6 +331,7 @@ int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void
     a.B = p->B; a.H = p->H; a.T = p->T; a.d = p->d; a.m = tc_mf(p->m); a.m_real = p->m; a.omega_ld = p->m; a.state_m = p->m; a.p_off = 0; a.W = p->W;
     a.omega_stride = p->omega_per_head ? (long)p->d * p->m : 0;
     a.chunks_per_cta = 16;
+    a.log2_eps_m = p->eps > 0.f ? (float)(log2((double)p->eps) + log2((double)p->m)) : -INFINITY;
     // the forward of the same parameters ran on the same kernels, so its boundary images can be taken over
     a.reuse_state = (p->flags & LINSIMP_FLAG_REUSE_FWD_STATE) && use_tc(p, LINSIMP_OP_FWD);
     a.q = q; a.k = k; a.v = v; a.r = r; a.u = u; a.omega = omega;

@@ -36,6 +36,12 @@ static constexpr int BC = kTcChunk;         // 16 tokens per chunk
 static constexpr int BNT = 512;
 static constexpr int BR = 4;                 // threads per tile row / output channel
 
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float ex2a(float x)
 {
     float y;
@@ -87,8 +93,8 @@ struct BwdTcSmem {
     static constexpr int OFF_DNH = OFF_DOH + BC * ROWB;         // [17][D] bf16: dN = dO/den rounded, row 16 = zeros
     static constexpr int OFF_AQ = OFF_DNH + (BC + 1) * ROWB;    // [16][MF] fp32: a_i = a_b + sum_{j<=i} chi'_j
     static constexpr int OFF_ROWS = OFF_AQ + BC * MF * 4;       // hn partial [4][128], -sum dl [128]
-    static constexpr int OFF_SC = OFF_ROWS + 5 * 128 * 4;       // 1/den[16], L[16], partial dots [16 warps], dZ[16]
-    static constexpr int TOTAL = OFF_SC + 256;
+    static constexpr int OFF_SC = OFF_ROWS + 5 * 128 * 4;       // 1/den[16], L[16], normaliser guard [16], dZ[16]
+    static constexpr int TOTAL = OFF_SC + 256 + 128;            // + the warps' partial sums [16][2]
 };
 
 // TMEM column map (512 allocated)
@@ -118,7 +124,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
          float *__restrict__ dv_intra, float *__restrict__ dchi_intra, int *__restrict__ status,
          const float *__restrict__ delta_ext, int grad32, float *__restrict__ delta_out, const int *__restrict__ seq_lens,
          const bf16 *__restrict__ hist_r, const bf16 *__restrict__ hist_u, int n_hist_arg, float *__restrict__ dhr_acc,
-         float *__restrict__ dhu_acc)
+         float *__restrict__ dhu_acc, float log2_eps_m)
 {
     constexpr bool EXT = MODE == 1, DOT = MODE == 2, HIST = MODE == 3;
     const int n_hist = HIST ? n_hist_arg : 0;
@@ -186,15 +192,16 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
     // staging of the chunk's G^M block (MF * D * 4 bytes) over tile buffers that hold no zero padding in this instance
     uint8_t *gm_stage = (MF == 128) ? psi_s : (D == 128 ? xdg_s : psi_s);
     float *aq = (float *)(smem + S::OFF_AQ);          // [16][MF]
-    float *hnp = (float *)(smem + S::OFF_ROWS);       // [4][128]
+    float *hnp = (float *)(smem + S::OFF_ROWS);       // [4][128] the column quarters' parts of |x|^2/2, later of zeta
     float *sdlp = hnp + 512;                          // [128] minus the row sums of dl
-    float *sdpart = (float *)(smem + S::OFF_PM);      // [2][4][128] the column quarters' parts of psi'.dpsiN and of zeta,
+    float *sdpart = (float *)(smem + S::OFF_PM);      // [4][128] the column quarters' parts of psi'.dpsiN,
                                                       // over the masked pair weights (no product reads them any more)
     float *dqp = (float *)(smem + S::OFF_DQP);        // [4][2][128]
     float *invs = (float *)(smem + S::OFF_SC);        // [16] 1/den_i
     float *Ls = invs + 16;                            // [16]
-    float *dred = Ls + 16;                            // [16 warps] partial sums of psi' . dpsiN
-    float *dzs = dred + 16;                           // [16] dZ_i of the chunk's queries
+    float *epsq = Ls + 16;                            // [16] guard of the normaliser, eps m exp(-L_i)
+    float *dzs = epsq + 16;                           // [16] dZ_i of the chunk's queries
+    float *dred = dzs + 16;                           // [16 warps][2] partial sums of psi' . dpsiN and of zeta
 
     const uint32_t om_addr = smem_u32(smem + S::OFF_OM);
     const uint32_t mbt_addr = smem_u32(smem + S::OFF_CHUNK);
@@ -299,6 +306,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 if (ch == 0) {
                     invs[il] = inv;
                     Ls[il] = Lq;
+                    epsq[il] = ex2a(log2_eps_m - Lq * LOG2E);
                 }
             }
         }
@@ -633,24 +641,41 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     dot += d2.x + d2.y;
                 }
                 // the row's parts of psi' . dpsiN and of zeta: 1^T dl_ic = psi'.dpsiN + dZ_i zeta_ic needs no second pass
+                const float zrow = z2.x + z2.y;
                 sdpart[h * 128 + t] = dot;
-                sdpart[512 + h * 128 + t] = z2.x + z2.y;
-                dot = warp_sum(dot);
-                if (lane == 0) dred[warp] = dot;
+                hnp[h * 128 + t] = zrow;            // the |x|^2 partials kept there were consumed with the exponentials
+                {
+                    // both warp sums in one butterfly: the lower half of the warp collects the dots, the upper half zeta
+                    const bool lo = lane < 16;
+                    float acc = lo ? dot : zrow;
+                    acc += __shfl_xor_sync(0xffffffffu, lo ? zrow : dot, 16);
+#pragma unroll
+                    for (int sh = 8; sh > 0; sh >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, sh);
+                    if ((lane & 15) == 0) dred[warp * 2 + (lane >> 4)] = acc;
+                }
                 __syncthreads();
                 // rows of query qi sit in the warps with bit 1 of the warp index equal to qi
                 const int qi = t >> 6;
-                float dsum = 0.f;
+                float dsum = 0.f, zsum = 0.f;
 #pragma unroll
-                for (int w8 = 0; w8 < 8; ++w8) dsum += dred[(w8 >> 1) * 4 + qi * 2 + (w8 & 1)];
+                for (int w8 = 0; w8 < 8; ++w8) {
+                    const float2 part = *(const float2 *)(dred + 2 * ((w8 >> 1) * 4 + qi * 2 + (w8 & 1)));
+                    dsum += part.x;
+                    zsum += part.y;
+                }
                 if (EXT) dsum = (i < T) ? delta_ext[(long)bh * T + i] : 0.f;
                 if (DOT && (t & 63) == 0 && h == 0 && i < T) atomicAdd(delta_out + (long)bh * T + i, dsum);
-                const float dz = -dsum * invs[il];
+                // dZ_i = -(dN_i . N'_i) / den'_i.  The normaliser is the one these very operands give, den'_i = sum_c
+                // zeta_ic + eps m exp(-L_i), not the forward's: the numerator and normaliser parts of the key gradients
+                // cancel, and what is left of them is only as exact as the two are consistent with each other.
+                float dz;
+                if (EXT || DOT) dz = -dsum * invs[il];
+                else dz = -dsum * rcp_approx(fmaxf(zsum + epsq[il], 1e-37f));
                 if ((t & 63) == 0 && h == 0) dzs[il] = dz;
                 // minus the row sum of dl, in a fixed order (bit-reproducible); read by the dx epilogue after the next barrier
                 if (h == 0)
                     sdlp[t] = -((((sdpart[t] + sdpart[128 + t]) + sdpart[256 + t]) + sdpart[384 + t]) +
-                                dz * (((sdpart[512 + t] + sdpart[640 + t]) + sdpart[768 + t]) + sdpart[896 + t]));
+                                dz * (((hnp[t] + hnp[128 + t]) + hnp[256 + t]) + hnp[384 + t]));
                 if (!DOT)
 #pragma unroll
                 for (int hf = 0; hf < 2; ++hf) {
@@ -1648,7 +1673,7 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
             (const bf16 *)a.q, (const bf16 *)a.r, (const bf16 *)a.u, (const bf16 *)a.dO, a.L, a.lse,
             a.om_img, a.omega_stride != 0, a.H, a.T, a.W, NC, cpc, a.images, a.ab, (bf16 *)a.dq, a.dr_acc, a.du_acc,
             a.gstates, a.dv_intra, a.dchi_intra, a.status, a.delta_ext, a.grad32, a.delta_out, a.seq_lens,
-            (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist, a.dhr_acc, a.dhu_acc));
+            (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist, a.dhr_acc, a.dhu_acc, a.log2_eps_m));
     };
     if (a.delta_out) {
         launch(k_bwd_tc<D, MF, 2>);
