@@ -67,7 +67,7 @@ size_t tc_blocks_extra_bytes(int B, int H, int T, int d, int m, int op)
 {
     const size_t rows = (size_t)B * H * T, nb = m / kBlk;
     size_t n = nb * (up256(rows * d * 4) + 2 * up256(rows * 4));
-    if (op == 1) n = up256(rows * 4) + 3 * up256(rows * d * 4);
+    if (op == 1) n = up256(rows * 8) + 3 * up256(rows * d * 4);
     return n;
 }
 
@@ -85,7 +85,7 @@ void tc_blocks_carve(char *base, int B, int H, int T, int d, int m, int op, TcBl
     w->delta = nullptr;
     for (int x = 0; x < 5; ++x) w->g32[x] = nullptr;
     if (op == 1) {
-        w->delta = (float *)(base + off); off += up256(rows * 4);
+        w->delta = (float *)(base + off); off += up256(rows * 8);
         for (int x = 0; x < 3; ++x) {
             w->g32[x] = (float *)(base + off); off += up256(rows * d * 4);
         }
@@ -162,7 +162,7 @@ int tc_blocks_bwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float lo
     // first pass per block: the block's part of sum_c psi'_ic . dpsiN_ic (= dO_i . o_i den_i of the layer), from the
     // backward's own tile pipeline, added up over the blocks
     (void)log_eps_m;
-    cudaMemsetAsync(w.delta, 0, sizeof(float) * rows, st);
+    sc.check(cudaMemsetAsync(w.delta, 0, sizeof(float) * 2 * rows, st));
     // The workspace holds the boundary images of one block at a time.  Order of the passes: the first pass starts with
     // the last block (whose images the forward left behind, if the caller says so) and ends with block nb - 2; the
     // second pass starts there, on the images still in place.  Two of the 2 nb pre-passes are saved that way.
@@ -205,7 +205,7 @@ int tc_blocks_bwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float lo
 size_t tc_views_extra_bytes(int B, int H, int T, int d, int op)
 {
     const size_t rows = (size_t)B * H * T;
-    if (op == 1) return up256(rows * 4) + 5 * up256(rows * d * 4);
+    if (op == 1) return up256(rows * 8) + 5 * up256(rows * d * 4);
     return 2 * (up256(rows * d * 4) + 2 * up256(rows * 4));
 }
 
@@ -217,7 +217,7 @@ void tc_views_carve(char *base, int B, int H, int T, int d, int op, TcBlockWs *w
     w->delta = nullptr;
     for (int x = 0; x < 5; ++x) w->g32[x] = nullptr;
     if (op == 1) {
-        w->delta = (float *)(base + off); off += up256(rows * 4);
+        w->delta = (float *)(base + off); off += up256(rows * 8);
         for (int x = 0; x < 5; ++x) {
             w->g32[x] = (float *)(base + off); off += up256(rows * d * 4);
         }
@@ -264,7 +264,7 @@ int tc_views_bwd_run(const TcArgs &a, const TcBlockWs &w, cudaStream_t st)
 {
     LaunchScope sc = {st, 0};
     const long rows = (long)a.B * a.H * a.T, ntok = rows * a.d;
-    sc.check(cudaMemsetAsync(w.delta, 0, sizeof(float) * rows, st));
+    sc.check(cudaMemsetAsync(w.delta, 0, sizeof(float) * 2 * rows, st));
     for (int view = 0; view < 2; ++view) {
         TcArgs x = view_args(a, view);
         x.delta_out = w.delta;
@@ -278,6 +278,7 @@ int tc_views_bwd_run(const TcArgs &a, const TcBlockWs &w, cudaStream_t st)
     for (int view = 0; view < 2; ++view) {
         TcArgs x = view_args(a, view);
         x.delta_ext = w.delta;
+        x.log2_eps_m = a.log2_eps_m + 1.f;       // the combined normaliser carries the guard of both views
         x.grad32 = view == 0 ? 1 : 2;
         x.keep_acc = view == 1;
         x.hold_acc = 1;

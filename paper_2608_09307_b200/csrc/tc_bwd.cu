@@ -306,7 +306,9 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 if (ch == 0) {
                     invs[il] = inv;
                     Ls[il] = Lq;
-                    epsq[il] = ex2a(log2_eps_m - Lq * LOG2E);
+                    // guard of the normaliser in the units of the sum it joins: the block's shifted sums, or (EXT) the
+                    // layer's normaliser taken as 1
+                    epsq[il] = ex2a(log2_eps_m - (EXT ? pf_lse : Lq) * LOG2E);
                 }
             }
         }
@@ -663,13 +665,22 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     dsum += part.x;
                     zsum += part.y;
                 }
+                const long n_rows = (long)gridDim.y * T;              // the buffers hold [BH][T] sums, then [BH][T] normalisers
                 if (EXT) dsum = (i < T) ? delta_ext[(long)bh * T + i] : 0.f;
-                if (DOT && (t & 63) == 0 && h == 0 && i < T) atomicAdd(delta_out + (long)bh * T + i, dsum);
+                if (DOT && (t & 63) == 0 && h == 0 && i < T) {
+                    atomicAdd(delta_out + (long)bh * T + i, dsum);
+                    atomicAdd(delta_out + n_rows + (long)bh * T + i, zsum * invs[il]);
+                }
                 // dZ_i = -(dN_i . N'_i) / den'_i.  The normaliser is the one these very operands give, den'_i = sum_c
                 // zeta_ic + eps m exp(-L_i), not the forward's: the numerator and normaliser parts of the key gradients
                 // cancel, and what is left of them is only as exact as the two are consistent with each other.
+                // Where the layer is a sum over several calls (EXT), the first passes have added up the calls'
+                // normalisers relative to the forward's, sum_b zeta_b / den_fwd, and the forward's 1/den is corrected by it.
                 float dz;
-                if (EXT || DOT) dz = -dsum * invs[il];
+                if (EXT) {
+                    const float kappa = (i < T) ? delta_ext[n_rows + (long)bh * T + i] + epsq[il] : 1.f;
+                    dz = -dsum * invs[il] * rcp_approx(fmaxf(kappa, 1e-37f));
+                } else if (DOT) dz = 0.f;
                 else dz = -dsum * rcp_approx(fmaxf(zsum + epsq[il], 1e-37f));
                 if ((t & 63) == 0 && h == 0) dzs[il] = dz;
                 // minus the row sum of dl, in a fixed order (bit-reproducible); read by the dx epilogue after the next barrier

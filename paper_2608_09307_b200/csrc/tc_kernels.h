@@ -23,8 +23,9 @@ struct TcArgs {
     const float *omega;
     void *o;                         // forward: out; backward: in
     float *o32;                      // forward: when set, the output goes here in fp32 instead of o
-    const float *delta_ext;          // backward: when set, [BH][T] the layer's sum_c psi'_ic . dpsiN_ic to use instead of the block's own
-    float *delta_out;                // backward: when set, only that sum of this block is computed and added there (no gradients)
+    const float *delta_ext;          // backward: when set, [BH][T] the layer's sum_c psi'_ic . dpsiN_ic to use instead of the block's own,
+                                     // followed by [BH][T] the layer's normaliser relative to the forward's
+    float *delta_out;                // backward: when set, only those two sums of this block are computed and added there (no gradients)
     int keep_acc, hold_acc;          // backward: do not zero the dr / du accumulators first; do not convert them out at the end
     int grad32;                      // backward: dq, dk, dv point to fp32 buffers; 1 = write them, 2 = add to them
     float *L, *lse;
@@ -68,7 +69,7 @@ int tc_bwd_run(const TcArgs &a, cudaStream_t st);
 // over the features, so the blocks' results combine exactly).  Workspace pieces beyond the one-block layout:
 struct TcBlockWs {
     float *o32[4], *Lb[4], *lseb[4];   // per block: fp32 output, row shift, log-normaliser
-    float *delta;                      // backward: [BH][T] dO_i . o_i den_i of the whole layer
+    float *delta;                      // backward: [BH][T] dO_i . o_i den_i of the whole layer, then [BH][T] its normaliser relative to the forward's
     float *g32[5];                     // backward: dq, dk, dv (and, for the two views, dr, du) summed in fp32
 };
 int tc_blocks_supported(int d, int m);
