@@ -52,7 +52,7 @@
 extern "C" {
 #endif
 
-#define LINSIMP_VERSION 5
+#define LINSIMP_VERSION 6
 
 enum {
     LINSIMP_OK = 0,
@@ -91,7 +91,16 @@ enum {
      * the combined estimator (lse = log(m (Z1 + Z2 + 2 eps))), S_final / z_final the state of view 1.  Costs two
      * passes of the kernels.  bf16 I/O on the tensor-core kernels with m <= 128 only (LINSIMP_EUNSUPPORTED
      * otherwise); LINSIMP_FLAG_REUSE_FWD_STATE has no effect together with it. */
-    LINSIMP_FLAG_TWO_VIEWS = 4
+    LINSIMP_FLAG_TWO_VIEWS = 4,
+    /* linsimp_bwd (and the forward whose states it reuses), tensor-core kernels: the chunk-boundary states enter the
+     * backward's products as two bf16 terms instead of one.  The backward recomputes the output (App. C) from a
+     * bf16 operand image of M_b (Eq. Mstate); dZ_i sees that output, while every key's own value enters its gradient
+     * exactly, and the two cancel in dk (d l / d z = omega - z, App. C): the image's rounding is the largest part of
+     * the error of dk (up to 2.3e-2 of max|dk| on a few of 170 surveyed seeds; below 1e-2 with this bit).  Costs a
+     * second image per chunk in the workspace (linsimp_workspace_bytes accounts for it) and about a sixth more time in
+     * the backward's tile kernel.  A forward that is to leave its states for LINSIMP_FLAG_REUSE_FWD_STATE must be
+     * given the bit as well.  No effect on the fp32 kernels, whose state is exact. */
+    LINSIMP_FLAG_STATE_TWO_TERMS = 8
 };
 
 typedef struct {

@@ -10,6 +10,7 @@ ALGO_DEFAULT, ALGO_FP32 = 0, 1
 FLAG_REUSE_FWD_STATE = 1
 FLAG_OMEGA_IMAGE = 2
 FLAG_TWO_VIEWS = 4
+FLAG_STATE_TWO_TERMS = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblinsimp.so")
@@ -167,10 +168,12 @@ def last_launch_count(op):
 
 
 def fwd(q, k, v, r, u, omega, W=64, eps=1e-30, algo=ALGO_DEFAULT, return_state=False, workspace=None,
-        out=None, stream=None, two_views=False):
+        out=None, stream=None, two_views=False, two_term_state=False):
     """linsimp_fwd.  q,k,v,r,u [B,H,T,d] (fp32 or bf16, CUDA); omega fp32 [d,m] or [H,d,m].
 
     two_views: both orientations of the trilinear score averaged (LINSIMP_FLAG_TWO_VIEWS).
+    two_term_state: leave the boundary states for a backward that is called with reuse_fwd_state and two_term_state
+    (LINSIMP_FLAG_STATE_TWO_TERMS; the workspace must have the size that backward asks for).
     Returns (o, rowmax_L, lse) and, with return_state, also (S_final, z_final).
     """
     lib = load_library()
@@ -178,7 +181,8 @@ def fwd(q, k, v, r, u, omega, W=64, eps=1e-30, algo=ALGO_DEFAULT, return_state=F
     B, H, T, d = q.shape
     m = omega.shape[-1]
     dv = v.shape[-1]
-    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps, FLAG_TWO_VIEWS if two_views else 0,
+    p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps,
+                    (FLAG_TWO_VIEWS if two_views else 0) | (FLAG_STATE_TWO_TERMS if two_term_state else 0),
                     0 if dv == d else dv)
     o = torch.empty_like(v) if out is None else out
     L = torch.empty((B, H, T), dtype=torch.float32, device=q.device)
@@ -284,8 +288,11 @@ def ring_fill(r, u, ring_r, ring_u, t_first=0, stream=None):
 
 
 def bwd(q, k, v, r, u, omega, o, L, lse, dO, W=64, eps=1e-30, algo=ALGO_DEFAULT, workspace=None, stream=None,
-        reuse_fwd_state=False, two_views=False):
+        reuse_fwd_state=False, two_views=False, two_term_state=False):
     """linsimp_bwd.  Returns dq, dk, dv, dr, du (same shape/dtype as the inputs).
+
+    two_term_state: the boundary states enter the backward's products as two bf16 terms (LINSIMP_FLAG_STATE_TWO_TERMS):
+    halves the error of dk for a sixth more time in the tile kernel and a second state image in the workspace.
 
     reuse_fwd_state: `workspace` is the tensor the preceding fwd() call on the same inputs was given
     (sized for the backward) and has not been written since; the backward then skips the state pre-pass.
@@ -298,8 +305,8 @@ def bwd(q, k, v, r, u, omega, o, L, lse, dO, W=64, eps=1e-30, algo=ALGO_DEFAULT,
         raise ValueError("reuse_fwd_state needs the workspace of the forward call")
     dv = v.shape[-1]
     p = make_params(B, H, T, d, m, W, _io_dtype(q), omega.dim() == 3, algo, eps,
-                    (FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0) | (FLAG_TWO_VIEWS if two_views else 0),
-                    0 if dv == d else dv)
+                    (FLAG_REUSE_FWD_STATE if reuse_fwd_state else 0) | (FLAG_TWO_VIEWS if two_views else 0) |
+                    (FLAG_STATE_TWO_TERMS if two_term_state else 0), 0 if dv == d else dv)
     grads = [torch.empty_like(x) for x in (q, k, v, r, u)]
     ws, ws_bytes = _workspace(p, OP_BWD, workspace, q.device)
     _check(lib.linsimp_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(r), _ptr(u), _ptr(omega),

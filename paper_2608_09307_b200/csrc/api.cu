@@ -86,7 +86,8 @@ bool params_ok(const linsimp_params *p, int op, bool dv_taken = false)
     if (p->io_dtype != LINSIMP_F32 && p->io_dtype != LINSIMP_BF16) return false;
     if (p->algo != LINSIMP_ALGO_DEFAULT && p->algo != LINSIMP_ALGO_FP32) return false;
     if (!(p->eps >= 0.f)) return false;
-    if (p->flags & ~(LINSIMP_FLAG_REUSE_FWD_STATE | LINSIMP_FLAG_OMEGA_IMAGE | LINSIMP_FLAG_TWO_VIEWS)) return false;
+    if (p->flags & ~(LINSIMP_FLAG_REUSE_FWD_STATE | LINSIMP_FLAG_OMEGA_IMAGE | LINSIMP_FLAG_TWO_VIEWS | LINSIMP_FLAG_STATE_TWO_TERMS))
+        return false;
     if ((p->flags & LINSIMP_FLAG_TWO_VIEWS) && !(op == LINSIMP_OP_FWD || op == LINSIMP_OP_BWD)) return false;
     return true;
 }
@@ -163,7 +164,7 @@ bool use_tc(const linsimp_params *p, int op)
 }
 
 struct TcLayout {
-    size_t status, chi_ml, segtot, images, ab, om_img, chi32, gstates, segsum, dv_intra, dchi_intra, dr_acc, du_acc, dhr_acc,
+    size_t status, chi_ml, segtot, images, ab, om_img, chi32, images_lo, gstates, segsum, dv_intra, dchi_intra, dr_acc, du_acc, dhr_acc,
         dhu_acc, total;
 };
 
@@ -194,6 +195,8 @@ TcLayout tc_layout(const linsimp_params *p, int op)
     if (op == LINSIMP_OP_BWD) {
         L.chi32 = off;                       // first, so that a forward given a backward-sized workspace can fill it
         off = align_up(off + BH * NC * kTcChunk * mf * sizeof(float), 1024);
+        L.images_lo = off;                   // second, for the same reason
+        if (p->flags & LINSIMP_FLAG_STATE_TWO_TERMS) off = align_up(off + BH * NC * (size_t)128 * mf * 2, 1024);
         L.gstates = off;
         off = align_up(off + BH * NC * E * sizeof(float), 1024);
         L.segsum = off;
@@ -300,7 +303,10 @@ int run_tc(const linsimp_params *p, const void *q, const void *k, const void *v,
     if (!state_only && use_tc(p, LINSIMP_OP_BWD)) {
         // a workspace of the backward's size: leave the fp32 key features where LINSIMP_FLAG_REUSE_FWD_STATE expects them
         const TcLayout LB = tc_layout(p, LINSIMP_OP_BWD);
-        if (workspace_bytes >= LB.total) a.chi32 = (float *)(ws + LB.chi32);
+        if (workspace_bytes >= LB.total) {
+            a.chi32 = (float *)(ws + LB.chi32);
+            if (p->flags & LINSIMP_FLAG_STATE_TWO_TERMS) a.images_lo = (uint8_t *)(ws + LB.images_lo);
+        }
     }
     if (cudaMemsetAsync(a.status, 0, 256, (cudaStream_t)stream) != cudaSuccess) return LINSIMP_ECUDA;
     const int op = state_only ? LINSIMP_OP_STATE : LINSIMP_OP_FWD;
@@ -345,6 +351,7 @@ int run_tc_bwd(const linsimp_params *p, const void *q, const void *k, const void
     a.ab = (float *)(tws + TL.ab);
     a.om_img = (uint8_t *)(tws + TL.om_img);
     a.chi32 = (float *)(tws + TL.chi32);
+    if (p->flags & LINSIMP_FLAG_STATE_TWO_TERMS) a.images_lo = (uint8_t *)(tws + TL.images_lo);
     a.gstates = (float *)(tws + TL.gstates);
     a.segsum = (float *)(tws + TL.segsum);
     a.dv_intra = (float *)(tws + TL.dv_intra);
@@ -392,6 +399,7 @@ int run_tc_views(int op, const linsimp_params *p, const void *q, const void *k, 
     a.om_img = (uint8_t *)(ws + L.om_img);
     if (op == LINSIMP_OP_BWD) {
         a.chi32 = (float *)(ws + L.chi32);
+        if (p->flags & LINSIMP_FLAG_STATE_TWO_TERMS) a.images_lo = (uint8_t *)(ws + L.images_lo);
         a.gstates = (float *)(ws + L.gstates);
         a.segsum = (float *)(ws + L.segsum);
         a.dv_intra = (float *)(ws + L.dv_intra);
@@ -439,6 +447,7 @@ int run_tc_blocks(int op, const linsimp_params *p, const void *q, const void *k,
         // (the forward of the same parameters leaves the last block's boundary images in place)
         a.reuse_state = (p->flags & LINSIMP_FLAG_REUSE_FWD_STATE) != 0;
         a.chi32 = (float *)(ws + L.chi32);
+        if (p->flags & LINSIMP_FLAG_STATE_TWO_TERMS) a.images_lo = (uint8_t *)(ws + L.images_lo);
         a.gstates = (float *)(ws + L.gstates);
         a.segsum = (float *)(ws + L.segsum);
         a.dv_intra = (float *)(ws + L.dv_intra);

@@ -36,6 +36,7 @@ static constexpr int BC = kTcChunk;         // 16 tokens per chunk
 static constexpr int BNT = 512;
 static constexpr int BR = 4;                 // threads per tile row / output channel
 
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 __device__ __forceinline__ float rcp_approx(float x)
 {
     float y;
@@ -114,7 +115,7 @@ __device__ __forceinline__ int anchor_of(int i, int x) { return i - ((i - x) & 6
 // MODE 3 (HIST) is the backward of a segment that continues a sequence: the anchors of the n_hist tokens before the
 // segment come from hist_r, hist_u, and what the segment's queries contribute to the gradients of those anchors
 // leaves through the accumulators dhr_acc, dhu_acc [BH][n_hist][D].
-template <int D, int MF, int MODE>
+template <int D, int MF, int MODE, bool TWO>
 __global__ void __launch_bounds__(BNT, 1)
 k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__restrict__ u,
          const bf16 *__restrict__ dO, const float *__restrict__ Lin, const float *__restrict__ lse,
@@ -124,7 +125,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
          float *__restrict__ dv_intra, float *__restrict__ dchi_intra, int *__restrict__ status,
          const float *__restrict__ delta_ext, int grad32, float *__restrict__ delta_out, const int *__restrict__ seq_lens,
          const bf16 *__restrict__ hist_r, const bf16 *__restrict__ hist_u, int n_hist_arg, float *__restrict__ dhr_acc,
-         float *__restrict__ dhu_acc, float log2_eps_m)
+         float *__restrict__ dhu_acc, float log2_eps_m, const uint8_t *__restrict__ images_lo)
 {
     constexpr bool EXT = MODE == 1, DOT = MODE == 2, HIST = MODE == 3;
     const int n_hist = HIST ? n_hist_arg : 0;
@@ -135,7 +136,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
     extern __shared__ __align__(1024) uint8_t smem_dyn[];
     // 1024-byte alignment by an offset into the array (not by pointer casts), so that accesses stay shared-space loads/stores
     uint8_t *smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-    __shared__ uint64_t bar_img, bar_om, bar_mma[10];
+    __shared__ uint64_t bar_img, bar_om, bar_mma[10], bar_lo, bar_omr, bar_aux;
     __shared__ uint32_t tmem_base_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -156,6 +157,9 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
         mbar_init(&bar_img, 1);
         mbar_init(&bar_om, 1);
         for (int x = 0; x < 10; ++x) mbar_init(&bar_mma[x], 1);
+        mbar_init(&bar_lo, 1);
+        mbar_init(&bar_omr, 1);
+        mbar_init(&bar_aux, 1);
         fence_barrier_init();
     }
     // the padding blocks of the psi tile (MF = 64) and of the dg tile (D = 64) must read as zero
@@ -176,6 +180,14 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
         tmem_st_wait();
     }
     const uint8_t *img_bh = images + (long)bh * NC * S::IMG_CHUNK;
+    // Second bf16 term of the boundary state (what the image's rounding leaves).  dZ_i sees the output the state
+    // operand gives, the keys' own values enter exactly, and the two cancel in the key gradients: the image alone
+    // leaves its rounding in dk.  No buffer is free for a second image, so it takes turns with Omega, which is read
+    // at the two ends of a tile only: in after the first product, out again after the last product that reads it.
+    static_assert(S::IMG_M == S::IMG_OM, "the second state term takes the Omega buffer");
+    constexpr bool use_lo = TWO;        // (compile-time: the one-term kernel carries none of this)
+    const uint8_t *lo_bh = use_lo ? images_lo + (long)bh * NC * S::IMG_M : nullptr;
+    const uint8_t *om_src = om_img + (long)(om_per_head ? bh % H : 0) * S::IMG_OM;
     if (tid == 0) {
         mbar_arrive_expect_tx(&bar_om, S::IMG_OM);
         bulk_g2s(smem + S::OFF_OM, om_img + (long)(om_per_head ? bh % H : 0) * S::IMG_OM, S::IMG_OM, &bar_om);
@@ -216,6 +228,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
     const uint32_t id_dp = make_idesc_f16(128, BC, 1, 0, 1);       // dg . V^T              (B MN-major)
     const uint32_t id_gm = make_idesc_f16(128, 160, 1, 1, 1);      // psi^T [dg | dPm | S]  (both MN-major)
     const uint32_t id_n16 = make_idesc_f16(128, BC, 1, 1, 1);      // dg^T Pm
+    const uint32_t id_dlo = make_idesc_f16(128, MF, 1, 0, 1);      // dg . Mb_lo^T, all features
     const uint32_t id_dpsih = make_idesc_f16(128, 64, 1, 0, 1);    // dg . Mb^T, dPm . chi' (B MN-major), 64 features
     const uint32_t id_dxh = make_idesc_f16(128, 64, 0, 1, 0);      // Omega . dl^T          (fp16, A MN-major), one query
 
@@ -417,6 +430,11 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     if (hf == 1) {
                         mbar_wait(&bar_mma[7], phase, status, 29);
                         tc_fence_after();
+                        if (tid == 0 && use_lo) {
+                            // the first product has read Omega: the buffer takes the state's second term
+                            mbar_arrive_expect_tx(&bar_lo, S::IMG_M);
+                            bulk_g2s(smem + S::OFF_OM, lo_bh + (long)n * S::IMG_M, S::IMG_M, &bar_lo);
+                        }
                     }
                     uint32_t v[CPT / 2];
                     if (CPT == 32) tmem_ld16(tm + lane_off + TB_MAIN + hf * (MF / 2) + h * (CPT / 2), (uint32_t(&)[16])v);
@@ -588,13 +606,25 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
             __syncthreads();
             if (tid == 0) {
                 tc_fence_after();
-                // second 64-feature block of dpsiN, over the second half of Gt (the du epilogue has read it)
+                // the state's second term for all features at once, dg . Mb_lo^T, over Gt (the du epilogue has read it):
+                // features 64.. share the accumulator of the block below, features 0..63 are added when dpsiN is read
+                const uint64_t ddg = make_smem_desc(xdg_addr, 0, 1024, kSw128);
+                if (use_lo) {
+                    mbar_wait(&bar_lo, phase, status, 32);
+                    tc_fence_after();
+                    const uint64_t dml = make_smem_desc(om_addr, 128 * 128, 1024, kSw128);
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_f16_ss(tm + TB_MAIN, desc_adv(ddg, (ks >> 2) * (128 * 128) + (ks & 3) * 32), desc_adv(dml, ks * 2048), id_dlo, ks > 0);
+                    tc_commit(&bar_aux);
+                }
+                // second 64-feature block of dpsiN
                 if (MF == 128) {
-                    const uint64_t ddg = make_smem_desc(xdg_addr, 0, 1024, kSw128), dmb = make_smem_desc(mbt_addr, 128 * 128, 1024, kSw128);
+                    const uint64_t dmb = make_smem_desc(mbt_addr, 128 * 128, 1024, kSw128);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
                         mma_f16_ss(tm + TB_MAIN + 64, desc_adv(ddg, (ks >> 2) * (128 * 128) + (ks & 3) * 32),
-                                   desc_adv(dmb, ks * 2048 + 128 * 128), id_dpsih, ks > 0);
+                                   desc_adv(dmb, ks * 2048 + 128 * 128), id_dpsih, use_lo || ks > 0);
                     mma_f16_ss(tm + TB_MAIN + 64, make_smem_desc(b3_addr, 0, 1024, kSw128),
                                make_smem_desc(chi_addr + BC * 128, BC * 128, 1024, kSw128), id_dpsih, 1);
                 }
@@ -612,6 +642,14 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     psk[o4] = pv.x; psk[o4 + 1] = pv.y; psk[o4 + 2] = pv.z; psk[o4 + 3] = pv.w;
                 }
             mbar_wait(&bar_mma[3], phase, status, 25);
+            if (use_lo) {
+                mbar_wait(&bar_aux, phase, status, 34);
+                if (tid == 0) {
+                    // the products that read the state's second term are done: Omega returns for dxT and the next tile
+                    mbar_arrive_expect_tx(&bar_omr, S::IMG_OM);
+                    bulk_g2s(smem + S::OFF_OM, om_src, S::IMG_OM, &bar_omr);
+                }
+            }
             tc_fence_after();
             {
                 uint32_t v[CPT];
@@ -628,6 +666,15 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     const uint32_t col = (f0 < 64) ? TB_AUX + f0 : TB_MAIN + f0;
                     if (CPT == 32) tmem_ld16(tm + lane_off + col, (uint32_t(&)[16])v[hf * (CPT / 2)]);
                     else tmem_ld8(tm + lane_off + col, (uint32_t(&)[8])v[hf * (CPT / 2)]);
+                    if (use_lo && f0 < 64) {
+                        uint32_t w[CPT / 2];
+                        if (CPT == 32) tmem_ld16(tm + lane_off + TB_MAIN + f0, (uint32_t(&)[16])w);
+                        else tmem_ld8(tm + lane_off + TB_MAIN + f0, (uint32_t(&)[8])w);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int x = 0; x < CPT / 2; ++x)
+                            v[hf * (CPT / 2) + x] = __float_as_uint(__uint_as_float(v[hf * (CPT / 2) + x]) + __uint_as_float(w[x]));
+                    }
                     tmem_ld_wait();
                     float2 d2 = make_float2(0.f, 0.f);
 #pragma unroll
@@ -711,6 +758,7 @@ k_bwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
             tc_fence_before();
             __syncthreads();
             if (tid == 0) {
+                if (use_lo) mbar_wait(&bar_omr, phase, status, 33);
                 tc_fence_after();
                 // dxT = Omega . dl^T  (OmegaT image read MN-major: rows = p, 64-wide a blocks), one query
                 // (64 tile rows) at a time so that the epilogue of the first starts under the second
@@ -1095,8 +1143,9 @@ k_bwd_kv_tc(const bf16 *__restrict__ v, int T, int NC, const float *__restrict__
                 for (int hh = 0; hh < 2; ++hh) {
                     const int j = g + hh * 8, p = n0 + nt * 8 + 2 * t;
                     const float2 cx = *(const float2 *)(chi + j * LDC + p);
-                    *(float2 *)(dlo + j * MF + p) = make_float2((c[nt][hh * 2] + es[p] + di[nt][hh].x) * cx.x,
-                                                                (c[nt][hh * 2 + 1] + es[p + 1] + di[nt][hh].y) * cx.y);
+                    // the intra-chunk part belongs to pair weights formed from the bf16 image of chi'
+                    *(float2 *)(dlo + j * MF + p) = make_float2(fmaf(c[nt][hh * 2] + es[p], cx.x, di[nt][hh].x * bf16_round(cx.x)),
+                                                                fmaf(c[nt][hh * 2 + 1] + es[p + 1], cx.y, di[nt][hh].y * bf16_round(cx.y)));
                 }
         }
         if (n0 < D) {
@@ -1328,7 +1377,8 @@ k_bwd_kv_tc5(const bf16 *__restrict__ v, int T, int NC, const float *__restrict_
             float *dlo = chi_dl + (((long)bh * NC + n) * BC + half * 8) * MF + row;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                dlo[(long)j * MF] = (__uint_as_float(a1[j]) + es + di[j]) * xc[j];
+                // the intra-chunk part belongs to pair weights formed from the bf16 image of chi'
+                dlo[(long)j * MF] = fmaf(__uint_as_float(a1[j]) + es, xc[j], di[j] * bf16_round(xc[j]));
                 const int tok = n * BC + half * 8 + j;
                 if (tok < T) dv[seq_off + (long)tok * D + row] = __float2bfloat16_rn(__uint_as_float(a2[j]) + iv[j]);
             }
@@ -1684,15 +1734,24 @@ static int bwd_tc_impl(const TcArgs &a, cudaStream_t st)
             (const bf16 *)a.q, (const bf16 *)a.r, (const bf16 *)a.u, (const bf16 *)a.dO, a.L, a.lse,
             a.om_img, a.omega_stride != 0, a.H, a.T, a.W, NC, cpc, a.images, a.ab, (bf16 *)a.dq, a.dr_acc, a.du_acc,
             a.gstates, a.dv_intra, a.dchi_intra, a.status, a.delta_ext, a.grad32, a.delta_out, a.seq_lens,
-            (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist, a.dhr_acc, a.dhu_acc, a.log2_eps_m));
+            (const bf16 *)a.hist_r, (const bf16 *)a.hist_u, a.n_hist, a.dhr_acc, a.dhu_acc, a.log2_eps_m, a.images_lo));
     };
+    const bool two = a.images_lo != nullptr;
     if (a.delta_out) {
-        launch(k_bwd_tc<D, MF, 2>);
+        if (two) launch(k_bwd_tc<D, MF, 2, true>);
+        else launch(k_bwd_tc<D, MF, 2, false>);
         return sc.result();                   // first pass of a feature block: only its part of the layer's dO . o
     }
-    if (a.delta_ext) launch(k_bwd_tc<D, MF, 1>);
-    else if (a.n_hist > 0) launch(k_bwd_tc<D, MF, 3>);
-    else launch(k_bwd_tc<D, MF, 0>);
+    if (a.delta_ext) {
+        if (two) launch(k_bwd_tc<D, MF, 1, true>);
+        else launch(k_bwd_tc<D, MF, 1, false>);
+    } else if (a.n_hist > 0) {
+        if (two) launch(k_bwd_tc<D, MF, 3, true>);
+        else launch(k_bwd_tc<D, MF, 3, false>);
+    } else {
+        if (two) launch(k_bwd_tc<D, MF, 0, true>);
+        else launch(k_bwd_tc<D, MF, 0, false>);
+    }
     // Segments of the key/value sweep: one wave of CTAs (two per SM) where the sequence is long enough, never shorter
     // than KV_SEG chunks (the workspace holds one partial sum per KV_SEG chunks).
     const int slots = 2 * sm_count();

@@ -260,13 +260,14 @@ k_prep_tc5(const bf16 *__restrict__ k, const bf16 *__restrict__ v, const float *
 // read from tensor memory, rounded to bf16 and written as the chunk's state operand image (exclusive prefix).  The
 // operands arrive through a ring of bulk-copy stages; reading, converting and storing the image of chunk n overlaps
 // the products of chunk n.  Threads 0..63 carry the normaliser's prefix of the block's features.
-static constexpr int ST_STAGES = 6;
-template <int D, int MF>
+static constexpr int ST_STAGES = 6, ST_STAGES_TWO = 4;       // (with the second image to assemble, fewer stages fit two CTAs per SM)
+template <int D, int MF, bool TWO>
 struct StateSmem {
     static constexpr int VT = 128 * 32, CB = TC_C * 128;       // V^T image; one 64-feature block of a chi' image
     static constexpr int STAGE = VT + 3 * CB;
     static constexpr int OBUF = 128 * 128;                     // one 64-feature block of a state image, as it lies in global memory
-    static constexpr int TOTAL = ST_STAGES * STAGE + 2 * OBUF;
+    static constexpr int NST = TWO ? ST_STAGES_TWO : ST_STAGES;
+    static constexpr int TOTAL = NST * STAGE + (TWO ? 4 : 2) * OBUF;   // two buffers for the image (and two for its rounding remainder)
 };
 
 // The walk over a long sequence is cut into segments (blockIdx.z) so that enough CTAs run: a first launch (TOTALS)
@@ -274,18 +275,19 @@ struct StateSmem {
 // [BH][segments][MF/64][128*64 + 64] fp32; the second launch starts every segment from the sums of the segments before it.
 static constexpr int kStateSegMax = 8;
 static constexpr int kSegTot = 128 * 64 + 64;                  // floats per (unit, segment, feature block)
-template <int D, int MF, bool TOTALS>
+template <int D, int MF, bool TOTALS, bool TWO>
 __global__ void __launch_bounds__(256, 1)
 k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int NC, float *__restrict__ ab,
            float *__restrict__ S_final, float *__restrict__ z_final, int m_real, const float *__restrict__ S_init,
            const float *__restrict__ z_init, int state_m, int p_off, int *__restrict__ status, int seg_len,
-           float *__restrict__ segtot, int n_seg)
+           float *__restrict__ segtot, int n_seg, uint8_t *__restrict__ images_lo)
 {
     using G = TcGeom<D, MF>;
-    using SS = StateSmem<D, MF>;
+    using SS = StateSmem<D, MF, TWO>;
+    constexpr int NST = SS::NST;
     extern __shared__ __align__(1024) uint8_t smem_dyn[];
     uint8_t *smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
-    __shared__ uint64_t full[ST_STAGES], bar_mma;
+    __shared__ uint64_t full[NST], bar_mma;
     __shared__ uint32_t tmem_base_s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kb = blockIdx.x, bh = blockIdx.y, seg = blockIdx.z;
@@ -297,7 +299,7 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
         tmem_relinquish();
     }
     if (tid == 0) {
-        for (int x = 0; x < ST_STAGES; ++x) mbar_init(&full[x], 1);
+        for (int x = 0; x < NST; ++x) mbar_init(&full[x], 1);
         mbar_init(&bar_mma, 1);
         fence_barrier_init();
     }
@@ -327,12 +329,14 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
         if (z_init && kb * 64 + na < m_real) arun = z_init[(long)bh * state_m + p_off + kb * 64 + na];
         for (int s2 = 0; s2 < seg; ++s2) arun += tot_bh[(long)s2 * (MF / 64) * kSegTot + 128 * 64 + na];
     }
-    uint8_t *obuf = smem + ST_STAGES * SS::STAGE;
+    uint8_t *obuf = smem + NST * SS::STAGE;
     uint8_t *img_bh = images + (long)bh * NC * G::IMG_CHUNK;
+    // second bf16 term of the state (what the rounding of the image leaves), same layout, for the backward (nullable)
+    uint8_t *lo_bh = (!TOTALS && TWO) ? images_lo + (long)bh * NC * G::IMG_M : nullptr;
     const uint8_t *ml_bh = chi_ml + (long)bh * NC * 2 * G::IMG_CHI;
     auto load = [&](int n) {                                     // (stages and barrier phases count from the segment's first chunk)
-        uint8_t *st = smem + ((n - n_begin) % ST_STAGES) * SS::STAGE;
-        uint64_t *bar = &full[(n - n_begin) % ST_STAGES];
+        uint8_t *st = smem + ((n - n_begin) % NST) * SS::STAGE;
+        uint64_t *bar = &full[(n - n_begin) % NST];
         const uint8_t *img = img_bh + (long)n * G::IMG_CHUNK;
         const uint8_t *ml = ml_bh + (long)n * 2 * G::IMG_CHI;
         mbar_arrive_expect_tx(bar, SS::STAGE);
@@ -342,29 +346,32 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
         bulk_g2s(st + SS::VT + 2 * SS::CB, ml + G::IMG_CHI + kb * SS::CB, SS::CB, bar);
     };
     if (tid == 0)
-        for (int n = n_begin; n < n_begin + ST_STAGES && n < n_end; ++n) load(n);
+        for (int n = n_begin; n < n_begin + NST && n < n_end; ++n) load(n);
     const uint32_t idesc = make_idesc_f16(128, 64, 1, 0, 1);     // bf16; A K-major (V^T rows of 16 tokens), B MN-major
     tc_fence_before();
     __syncthreads();                                             // initial state in tensor memory before the first product
     tc_fence_after();
     uint32_t mma_phase = 0;
     for (int n = n_begin; n < n_end; ++n) {
-        const int sidx = (n - n_begin) % ST_STAGES;
+        const int sidx = (n - n_begin) % NST;
         uint8_t *st = smem + sidx * SS::STAGE;
         // the state before chunk n
         if (!TOTALS) {
             tmem_ld32(tm + lane_off + ch * 32, v);
             tmem_ld_wait();
         }
-        mbar_wait(&full[sidx], ((n - n_begin) / ST_STAGES) & 1, status, 30);
+        mbar_wait(&full[sidx], ((n - n_begin) / NST) & 1, status, 30);
         // the image buffer about to be rewritten was handed to a bulk store an iteration ago: its reads must be over
         if (!TOTALS && tid == 0) bulk_wait_read<0>();
         tc_fence_before();
         __syncthreads();                       // every thread holds its part of the state; stage n is in shared memory
         if (tid == 0) {
             // the image of the chunk before is complete in shared memory (written before the barrier): one bulk store
-            if (!TOTALS && n > n_begin)
+            if (!TOTALS && n > n_begin) {
                 bulk_s2g(img_bh + (long)(n - 1) * G::IMG_CHUNK + kb * SS::OBUF, obuf + ((n - 1 - n_begin) & 1) * SS::OBUF, SS::OBUF);
+                if (TWO && !TOTALS)
+                    bulk_s2g(lo_bh + (long)(n - 1) * G::IMG_M + kb * SS::OBUF, obuf + (2 + ((n - 1 - n_begin) & 1)) * SS::OBUF, SS::OBUF);
+            }
             tc_fence_after();
             const uint64_t da = make_smem_desc(smem_u32(st), 0, 256, kSw32);
 #pragma unroll
@@ -373,7 +380,7 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
             tc_commit(&bar_mma);
             // the stage of chunk n - 1 is free: its products have completed (waited for at the end of the iteration
             // before) and its reads for the normaliser lie before the barrier above
-            if (n > n_begin && n - 1 + ST_STAGES < n_end) load(n - 1 + ST_STAGES);
+            if (n > n_begin && n - 1 + NST < n_end) load(n - 1 + NST);
         }
         // the chunk's state operand image: row e, features [64 kb + 32 ch, + 32) = four 16-byte pieces
         // (assembled in shared memory in its final layout and stored as one contiguous 16 KB block: a row per thread
@@ -386,6 +393,14 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
 #pragma unroll
                 for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(__uint_as_float(v[i * 8 + 2 * x]), __uint_as_float(v[i * 8 + 2 * x + 1]));
                 *(uint4 *)(dst + sw_off<128>(e, ch * 4 + i)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                if (TWO && !TOTALS) {
+                    uint32_t pl[4];
+#pragma unroll
+                    for (int x = 0; x < 4; ++x)
+                        pl[x] = pack_bf16(__uint_as_float(v[i * 8 + 2 * x]) - __uint_as_float(pk[x] << 16),
+                                          __uint_as_float(v[i * 8 + 2 * x + 1]) - __uint_as_float(pk[x] & 0xffff0000u));
+                    *(uint4 *)(dst + 2 * SS::OBUF + sw_off<128>(e, ch * 4 + i)) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                }
             }
             fence_proxy_async_smem();
         }
@@ -409,8 +424,11 @@ k_state_tc(uint8_t *__restrict__ images, const uint8_t *__restrict__ chi_ml, int
     if (!TOTALS) {
         __syncthreads();                       // the last chunk's image is complete in shared memory
         if (tid == 0) {
-            if (n_end > n_begin)
+            if (n_end > n_begin) {
                 bulk_s2g(img_bh + (long)(n_end - 1) * G::IMG_CHUNK + kb * SS::OBUF, obuf + ((n_end - 1 - n_begin) & 1) * SS::OBUF, SS::OBUF);
+                if (TWO && !TOTALS)
+                    bulk_s2g(lo_bh + (long)(n_end - 1) * G::IMG_M + kb * SS::OBUF, obuf + (2 + ((n_end - 1 - n_begin) & 1)) * SS::OBUF, SS::OBUF);
+            }
             bulk_wait_all<0>();
         }
     }
@@ -1085,7 +1103,6 @@ static int fwd_tc_impl(const TcArgs &a, cudaStream_t st)
             (const bf16 *)a.k, (const bf16 *)a.v, a.omega, a.omega_stride, a.m_real, a.omega_ld, a.H, a.T, NC, a.chi_ml, a.images,
             a.chi32, a.seq_lens, a.status));
     }
-    using SS = StateSmem<D, MF>;
     // segments of the state walk: as many as fill the two CTA slots of every SM, at most kStateSegMax, none for short
     // sequences
     int n_seg = (2 * sm_count()) / (BH * (MF / 64));
@@ -1095,15 +1112,20 @@ static int fwd_tc_impl(const TcArgs &a, cudaStream_t st)
     const int seg_len = (NC + n_seg - 1) / n_seg;
     n_seg = (NC + seg_len - 1) / seg_len;
     if (n_seg > 1) {
-        sc.check(cudaFuncSetAttribute(k_state_tc<D, MF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SS::TOTAL + 1024));
-        LS_LAUNCH(sc, "state_totals_tc", k_state_tc<D, MF, true><<<dim3(MF / 64, BH, n_seg - 1), 256, SS::TOTAL + 1024, st>>>(
+        using SS = StateSmem<D, MF, false>;
+        sc.check(cudaFuncSetAttribute(k_state_tc<D, MF, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SS::TOTAL + 1024));
+        LS_LAUNCH(sc, "state_totals_tc", k_state_tc<D, MF, true, false><<<dim3(MF / 64, BH, n_seg - 1), 256, SS::TOTAL + 1024, st>>>(
             a.images, a.chi_ml, NC, a.ab, nullptr, nullptr, a.m_real, nullptr, nullptr, a.state_m, a.p_off, a.status, seg_len,
-            a.segtot, n_seg));
+            a.segtot, n_seg, nullptr));
     }
-    sc.check(cudaFuncSetAttribute(k_state_tc<D, MF, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SS::TOTAL + 1024));
-    LS_LAUNCH(sc, "state_tc", k_state_tc<D, MF, false><<<dim3(MF / 64, BH, n_seg), 256, SS::TOTAL + 1024, st>>>(
-        a.images, a.chi_ml, NC, a.ab, a.S_final, a.z_final, a.m_real, a.S_init, a.z_init, a.state_m, a.p_off, a.status, seg_len,
-        a.segtot, n_seg));
+    auto walk = [&](auto kern, int smem_bytes) {
+        sc.check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes));
+        LS_LAUNCH(sc, "state_tc", kern<<<dim3(MF / 64, BH, n_seg), 256, smem_bytes, st>>>(
+            a.images, a.chi_ml, NC, a.ab, a.S_final, a.z_final, a.m_real, a.S_init, a.z_init, a.state_m, a.p_off, a.status, seg_len,
+            a.segtot, n_seg, a.images_lo));
+    };
+    if (a.images_lo) walk(k_state_tc<D, MF, false, true>, StateSmem<D, MF, true>::TOTAL + 1024);
+    else walk(k_state_tc<D, MF, false, false>, StateSmem<D, MF, false>::TOTAL + 1024);
     if (a.state_only) return sc.result();
     const int smem = S::TOTAL + 1024;
     const int cpc = a.chunks_per_cta;

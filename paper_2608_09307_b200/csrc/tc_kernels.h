@@ -42,6 +42,8 @@ struct TcArgs {
     uint8_t *chi_ml;                 // [BH][NC][2][16*m*2] the second and third bf16 term of chi' (chi' operand image layout)
     uint8_t *images;                 // [BH][NC][tc_image_bytes] operand images
     float *ab;                       // [BH][NC][m] exclusive boundary normalisers
+    uint8_t *images_lo;              // [BH][NC][128 x m] bf16 (nullable): what the bf16 rounding of each boundary state image leaves,
+                                     // in the image's layout; written by the pre-pass for the backward's second state term
     float *chi32;                    // [BH][NC*16][m] fp32 key features chi' (nullable): written by the pre-pass for the
                                      // backward's key/value sweep, which turns it into dl^k in place
     uint8_t *om_img;                 // [n_omega][m*d*2] OmegaT fp16 image

@@ -27,7 +27,7 @@ def test_exports_every_declared_symbol():
     for name in decl:
         assert hasattr(lib, name), name
     assert set(binding.EXPORTS) <= decl
-    assert lib.linsimp_version() == 5
+    assert lib.linsimp_version() == 6
 
 
 def test_workspace_and_argument_checks_on_host():
