@@ -351,7 +351,34 @@ def bench_secondary(P, synth, torch, dev, steps, peaks):
     tfw = flw / (msw * 1e-3) / 1e12
     win = dict(ms=msw, tokens_per_s=Bw * Tw / (msw * 1e-3), tflops=tfw, finite=bool(torch.isfinite(ow.float()).all()), **frac(tfw))
     del qw, kw, rw, vw, uw, ow
-    return dict(steps=steps,
+    # the main workload's step with the boundary states as two bf16 terms in the backward (LINSIMP_FLAG_STATE_TWO_TERMS)
+    def rms():
+        x = torch.randn(Bw, Hw, Tw, dw, device=dev, generator=gen)
+        return (x / x.pow(2).mean(dim=-1, keepdim=True).sqrt()).to(torch.bfloat16)
+
+    tq, tk, tv, tr, tu, tdo = (rms() for _ in range(6))
+    tom = torch.randn(dw, WORKLOAD["m"], device=dev, generator=gen)
+    pt = P.binding.make_params(Bw, Hw, Tw, dw, WORKLOAD["m"], WORKLOAD["W"], P.BF16, flags=P.binding.FLAG_STATE_TWO_TERMS)
+    wst = torch.empty(P.workspace_bytes(pt, P.OP_BWD), dtype=torch.uint8, device=dev)
+
+    def step_t():
+        o_, L_, lse_ = P.fwd(tq, tk, tv, tr, tu, tom, W=WORKLOAD["W"], workspace=wst, two_term_state=True)
+        P.bwd(tq, tk, tv, tr, tu, tom, o_, L_, lse_, tdo, W=WORKLOAD["W"], workspace=wst, reuse_fwd_state=True,
+              two_term_state=True)
+
+    for _ in range(3):
+        step_t()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step_t()
+    e1.record()
+    torch.cuda.synchronize()
+    two = dict(ms_per_step=e0.elapsed_time(e1) / steps, workspace_bytes=int(wst.numel()))
+    del tq, tk, tv, tr, tu, tdo, wst
+    return dict(steps=steps, two_term_state="main workload, fwd+bwd, boundary states as two bf16 terms in the backward",
+                c3_two_term_state=two,
                 exact_windowed="exact 512 x 32 windowed 2-simplicial layer on B=%d H=%d T=%d d=%d bf16, fwd only "
                                "(warp-level MMAs)" % (Bw, Hw, Tw, dw), winsimp=win,
                 c4_sweep="C4: B=4 H=8 T=8192 d=64 W=64 bf16, fwd+bwd, TFLOP/s in the 3x convention", c4=rows,
