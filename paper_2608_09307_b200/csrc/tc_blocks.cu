@@ -164,12 +164,13 @@ int tc_blocks_bwd_run(const TcArgs &a, int m_total, const TcBlockWs &w, float lo
     // backward's own tile pipeline, added up over the blocks
     (void)log_eps_m;
     sc.check(cudaMemsetAsync(w.delta, 0, sizeof(float) * 2 * rows, st));
-    // The workspace holds the boundary images of one block at a time.  Order of the passes: the first pass ends with
-    // block nb - 2 and the second pass starts there, on the images still in place, which saves one of the 2 nb pre-passes.
+    // The workspace holds the boundary images of one block at a time.  Order of the passes: the first pass starts with
+    // the last block (whose images the forward left behind, if the caller says so) and ends with block nb - 2; the
+    // second pass starts there, on the images still in place.  Two of the 2 nb pre-passes are saved that way.
     for (int i = 0; i < nb; ++i) {
         const int b = (i == 0) ? nb - 1 : i - 1;
         TcArgs x = block_args(a, m_total, b);
-        x.reuse_state = 0;                  // (the forward's block passes leave no second state term behind)
+        x.reuse_state = (i == 0) && a.reuse_state && !a.images_lo;   // (the forward's block passes leave no second state term behind)
         x.delta_out = w.delta;
         const int c = tc_bwd_run(x, st);
         if (c < 0) return c;
