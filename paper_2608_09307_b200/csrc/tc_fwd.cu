@@ -522,19 +522,11 @@ struct FwdWsSmem {
 // channel warps' private window of u (bf16 pairs, written twice 40 columns apart so that any 33 consecutive pairs are
 // contiguous).
 static constexpr uint32_t WS_X = 0, WS_L = 128, WS_P = 384, WS_U = 416;
-#ifndef LS_FWD_RS
-#define LS_FWD_RS 2
-#endif
-#ifndef LS_FWD_XE
-#define LS_FWD_XE 0
-#endif
-#ifndef LS_FWD_P1
-#define LS_FWD_P1 16       // columns requested per wait in the maximum pass
-#endif
-#ifndef LS_FWD_P2
-#define LS_FWD_P2 0        // 1: the exponential pass requests the next piece before working on the current one
-#endif
-static constexpr int WS_RS = LS_FWD_RS;        // threads per tile row in the row warps (1 or 2)
+// Settings of the row warps (each the better of the alternatives that were timed on the main workload).
+static constexpr bool WS_X_EARLY = false;      // the next tile's X before the mask (true) or after it (false)
+static constexpr int WS_MAX_COLS = 16;         // columns requested per wait in the maximum pass
+static constexpr bool WS_EXP_AHEAD = false;    // the exponential pass requests the next piece before working on the current one
+static constexpr int WS_RS = 2;                // threads per tile row in the row warps (1 or 2)
 static constexpr int WS_GW = 4 * WS_RS;        // warps of one row group
 static constexpr int WS_CW0 = 2 * WS_GW;       // first channel warp; then the product warp and the load warp
 static constexpr int WS_NT = (WS_CW0 + 8) * 32;   // (the last warpgroup: product warp, load warp, two idle warps)
@@ -704,7 +696,7 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 {
                     // (all of this thread's columns are requested before the one wait: a tensor-memory round trip per
                     // piece would dominate the pass)
-                    constexpr int PW = FH > LS_FWD_P1 ? LS_FWD_P1 : FH;  // columns per batch of loads
+                    constexpr int PW = FH > WS_MAX_COLS ? WS_MAX_COLS : FH;  // columns per batch of loads
                     float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int c0 = 0; c0 < FH; c0 += PW) {
@@ -737,14 +729,14 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 {
                     // pieces of 16 columns; the next piece is requested before the current one is worked on
                     uint32_t lv[2][16];
-                    if (LS_FWD_P2) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH, lv[0]);
+                    if (WS_EXP_AHEAD) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH, lv[0]);
 #pragma unroll
                     for (int pc = 0; pc < FH / 16; ++pc) {
                         const int c0 = pc * 16;
-                        if (!LS_FWD_P2) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0, lv[0]);
+                        if (!WS_EXP_AHEAD) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0, lv[0]);
                         tmem_ld_wait();
-                        if (LS_FWD_P2 && pc + 1 < FH / 16) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0 + 16, lv[(pc + 1) & 1]);
-                        const uint32_t *lc = lv[LS_FWD_P2 ? (pc & 1) : 0];
+                        if (WS_EXP_AHEAD && pc + 1 < FH / 16) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH + c0 + 16, lv[(pc + 1) & 1]);
+                        const uint32_t *lc = lv[WS_EXP_AHEAD ? (pc & 1) : 0];
 #pragma unroll
                         for (int c8 = 0; c8 < 2; ++c8) {
                             uint32_t pk[4];
@@ -774,7 +766,7 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                     if (tile + 2 >= NT) mbar_arrive(&bar_rowsfree[c & 1]);
                 }
                 // ---- the next tile's X (either here, while the pair weights of this one are being computed, or after the mask)
-                if (LS_FWD_XE) {
+                if (WS_X_EARLY) {
                     if (tile + 2 < NT) {
                         make_x(n, tile + 2, k + 1);
                     } else if (n + 1 < n_end) {
@@ -814,7 +806,7 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_pm[b]);
-                if (!LS_FWD_XE) {
+                if (!WS_X_EARLY) {
                     if (tile + 2 < NT) {
                         make_x(n, tile + 2, k + 1);
                     } else if (n + 1 < n_end) {

@@ -75,6 +75,15 @@ def test_workspace_and_argument_checks_on_host():
     assert P.workspace_bytes(two, P.OP_DECODE) == 0
     assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 128, 64, P.F32, flags=binding.FLAG_TWO_VIEWS), P.OP_FWD) == 0
     assert P.workspace_bytes(binding.make_params(2, 3, 100, 64, 256, 64, P.BF16, flags=binding.FLAG_TWO_VIEWS), P.OP_FWD) == 0
+    # the state as two bf16 terms: a second image (128 x m bf16) per 16-token chunk in the backward's workspace, none
+    # in the forward's; fp32 streams take the bit without effect
+    terms = binding.make_params(2, 3, 100, 64, 128, 64, P.BF16, flags=binding.FLAG_STATE_TWO_TERMS)
+    extra = P.workspace_bytes(terms, P.OP_BWD) - P.workspace_bytes(p, P.OP_BWD)
+    assert 2 * 3 * 7 * 128 * 128 * 2 <= extra < 2 * 3 * 7 * 128 * 128 * 2 + 4096
+    assert P.workspace_bytes(terms, P.OP_FWD) == P.workspace_bytes(p, P.OP_FWD)
+    f32 = binding.make_params(2, 3, 100, 64, 128, 64, P.F32)
+    f32t = binding.make_params(2, 3, 100, 64, 128, 64, P.F32, flags=binding.FLAG_STATE_TWO_TERMS)
+    assert P.workspace_bytes(f32t, P.OP_BWD) == P.workspace_bytes(f32, P.OP_BWD) > 0
     # normalisation / gate calls: one float per 128 rows of a unit, rounded up to 256 bytes
     assert P.workspace_bytes(p, P.OP_NORM) == 256
     big = binding.make_params(2, 16, 16384, 128, 128, 64, P.BF16)
