@@ -34,21 +34,22 @@ def _gpu_rows(x, units, lo, hi):
     return np.stack([to64(x[b_, h_, lo:hi]) for b_, h_ in units])
 
 
-def _run(cfg_name, with_bwd):
+def _run(cfg_name, with_bwd, two_term_state=False):
     cfg, t = synth.make_config(cfg_name, with_dO=with_bwd)
     g = {k_: v_.cuda() for k_, v_ in t.items()}
-    p = P.binding.make_params(cfg["B"], cfg["H"], cfg["T"], cfg["d"], cfg["m"], W, P.BF16)
+    p = P.binding.make_params(cfg["B"], cfg["H"], cfg["T"], cfg["d"], cfg["m"], W, P.BF16,
+                              flags=P.binding.FLAG_STATE_TWO_TERMS if two_term_state else 0)
     need = P.workspace_bytes(p, P.OP_FWD)
     if with_bwd:
         need = max(need, P.workspace_bytes(p, P.OP_BWD))
     ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
-    o, L, lse = P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], g["omega"], W=W, workspace=ws)
+    o, L, lse = P.fwd(g["q"], g["k"], g["v"], g["r"], g["u"], g["omega"], W=W, workspace=ws, two_term_state=two_term_state)
     assert P.binding.read_status(ws) == 0
     grads = None
     if with_bwd:
         # the launch configuration the benchmark times: the backward takes the boundary states over from the forward
         grads = P.bwd(g["q"], g["k"], g["v"], g["r"], g["u"], g["omega"], o, L, lse, g["dO"], W=W, workspace=ws,
-                      reuse_fwd_state=True)
+                      reuse_fwd_state=True, two_term_state=two_term_state)
         assert P.binding.read_status(ws) == 0
     torch.cuda.synchronize()
     assert torch.isfinite(o.float()).all()
@@ -66,8 +67,9 @@ def test_c2_layer_forward():
         assert e <= 2e-2, (lo, e)
 
 
-def test_c3_long_context_forward_backward():
-    cfg, t, o, grads = _run("C3", True)
+@pytest.mark.parametrize("two_term_state", [False, True])
+def test_c3_long_context_forward_backward(two_term_state):
+    cfg, t, o, grads = _run("C3", True, two_term_state)
     om = to64(t["omega"])
     T = cfg["T"]
     units = [(0, 3), (1, 12)]
@@ -78,6 +80,7 @@ def test_c3_long_context_forward_backward():
     for name, got, ref in zip(("dq", "dk", "dv", "dr", "du"), grads, g_ref):
         assert torch.isfinite(got.float()).all(), name
         e = rel_err(_gpu_rows(got, units, lo, hi), ref)
+        print("two-term state" if two_term_state else "one-term state", name, "%.1e" % e)
         assert e <= 2e-2, (name, e)
     # a middle slice: o and dq need only the prefix state; dr, du of an anchor need its 64 queries
     lo, hi = 8192 - 256, 8192 + 256
