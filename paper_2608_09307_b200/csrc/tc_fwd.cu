@@ -744,8 +744,9 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                             for (int x = 0; x < 4; ++x) {
                                 const int col = hf * FH + c0 + c8 * 8 + x * 2;
                                 const float2 arg = ffma2(make_float2(__uint_as_float(lc[c8 * 8 + x * 2]), __uint_as_float(lc[c8 * 8 + x * 2 + 1])), l2e, nshift);
-                                // every fourth pair as a polynomial on the FMA pipes, the rest on the special-function unit
-                                const float2 pp = (x == 3) ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+                                // d = 128: every fourth pair as a polynomial on the FMA pipes, the rest on the special-function
+                                // unit; d = 64: all of them there (the polynomial brought nothing at that width)
+                                const float2 pp = (x == 3 && D != 64) ? ex2_poly2(arg) : make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
                                 if (x & 1) zeta3 = ffma2(pp, *(const float2 *)(abs_ + col), zeta3);
                                 else zeta2 = ffma2(pp, *(const float2 *)(abs_ + col), zeta2);
                                 pk[x] = pack_bf16(pp.x, pp.y);
