@@ -525,7 +525,6 @@ static constexpr uint32_t WS_X = 0, WS_L = 128, WS_P = 384, WS_U = 416;
 // Settings of the row warps (each the better of the alternatives that were timed on the main workload).
 static constexpr bool WS_X_EARLY = false;      // the next tile's X before the mask (true) or after it (false)
 static constexpr int WS_MAX_COLS = 16;         // columns requested per wait in the maximum pass
-static constexpr bool WS_EXP_AHEAD = false;    // the exponential pass requests the next piece before working on the current one
 static constexpr int WS_RS = 2;                // threads per tile row in the row warps (1 or 2)
 static constexpr int WS_GW = 4 * WS_RS;        // warps of one row group
 static constexpr int WS_CW0 = 2 * WS_GW;       // first channel warp; then the product warp and the load warp
@@ -727,8 +726,10 @@ k_fwd_tc(const bf16 *__restrict__ q, const bf16 *__restrict__ r, const bf16 *__r
                 const float2 l2e = make_float2(LOG2E, LOG2E), nshift = make_float2(-shift, -shift);
                 float2 zeta2 = make_float2(0.f, 0.f), zeta3 = make_float2(0.f, 0.f);
                 {
-                    // pieces of 16 columns; the next piece is requested before the current one is worked on
+                    // pieces of 16 columns; at d = 128 the next piece is requested before the current one is worked on
+                    // (at d = 64 that brought nothing)
                     uint32_t lv[2][16];
+                    constexpr bool WS_EXP_AHEAD = D == 128;
                     if (WS_EXP_AHEAD) tmem_ld16(tm + lane_off + WS_L + b * 128 + hf * FH, lv[0]);
 #pragma unroll
                     for (int pc = 0; pc < FH / 16; ++pc) {
